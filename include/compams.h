@@ -1,0 +1,204 @@
+/*
+ * compams.h - C ABI of the B200 (sm_100a) COMP-AMS optimizer-step library.
+ *
+ * The library runs ONE iteration of Algorithm 2 ("Distributed COMP-AMS with error feedback") of
+ * "On Distributed Adaptive Optimization with Gradient Compression" (Li, Karimi, Li, ICLR 2022)
+ * per call, with all n workers held as rows of [n, d] buffers on one GPU:
+ *
+ *   worker i (Algorithm 2, lines 7-8):   x_i = g_i + e_i;  g~_i = C(x_i);  e_i <- x_i - g~_i
+ *   server   (Algorithm 2, lines 12-16): gbar = (1/n) sum_i g~_i;
+ *                                        m <- b1 m + (1-b1) gbar;  v <- b2 v + (1-b2) gbar^2;
+ *                                        vhat <- max(vhat, v);  theta <- theta - lr m / sqrt(vhat + eps)
+ *
+ * C is Top-k (Definition 1) or Block-Sign (Definition 2), applied block by block, the blocks
+ * being a contiguous partition of [0, d) (Section 3.1: usually one block per network layer).
+ *
+ * Conventions
+ *   - "host" / "device" after a pointer says where the memory lives. No call takes ownership of
+ *     caller memory. All device work is enqueued on the handle's CUDA stream (default: the legacy
+ *     default stream); calls return without synchronising unless stated otherwise.
+ *   - Every call returns COMPAMS_OK (0) or a negative compams_status. Nothing aborts, throws or
+ *     prints. One handle may be used by one host thread at a time.
+ *   - All state is fp32. Every fp32 operation of the update is a separately rounded IEEE
+ *     operation (no fused multiply-add, IEEE sqrt and division, subnormals kept).
+ *   - Gradients must be finite. NaN/Inf make the Top-k selection undefined (no fault, but the
+ *     kept set is unspecified).
+ */
+#ifndef COMPAMS_H
+#define COMPAMS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct compams_context* compams_handle;
+
+/* Compressors (Section 3.1). */
+enum compams_compressor {
+    COMPAMS_TOPK = 0,      /* Definition 1, per block; k_b = clamp(floor(k_ratio * d_b), 1, d_b) */
+    COMPAMS_BLOCKSIGN = 1  /* Definition 2: sign(x_B) * ||x_B||_1 / d_B */
+};
+
+enum compams_status {
+    COMPAMS_OK = 0,
+    COMPAMS_ERR_INVALID_ARG = -1,   /* a null pointer, a size out of range, malformed block offsets ... */
+    COMPAMS_ERR_ALLOC = -2,         /* host or device allocation failed */
+    COMPAMS_ERR_CUDA = -3,          /* a CUDA runtime call failed (see compams_last_cuda_error) */
+    COMPAMS_ERR_DEVICE_STATUS = -4  /* a kernel recorded an internal inconsistency in the status word */
+};
+
+/* Buffers readable through compams_get_buffer. */
+enum compams_buffer {
+    COMPAMS_BUF_E = 0,            /* float  [n, d]   error accumulators e_{t+1,i} (Algorithm 2, line 8)          */
+    COMPAMS_BUF_M = 1,            /* float  [d]      first moment m_t                                            */
+    COMPAMS_BUF_V = 2,            /* float  [d]      second moment v_t                                           */
+    COMPAMS_BUF_VHAT = 3,         /* float  [d]      running maximum vhat_t                                      */
+    COMPAMS_BUF_GBAR = 4,         /* float  [d]      averaged compressed gradient gbar_t                         */
+    COMPAMS_BUF_TOPK_IDX = 5,     /* int32  [n, K]   kept coordinates (index into [0, d)); K = sum_b k_b         */
+    COMPAMS_BUF_TOPK_VAL = 6,     /* float  [n, K]   kept values, bit-identical to x at that coordinate          */
+    COMPAMS_BUF_TOPK_SEG_OFFSETS = 7, /* int64 [M+1] block b of worker i owns entries [i*K+off[b], i*K+off[b+1]) */
+    COMPAMS_BUF_SIGN_BITS = 8,    /* uint32 [n, W]   Block-Sign sign bits, see below; W = sum_b ceil(d_b / 32)   */
+    COMPAMS_BUF_SIGN_WORD_OFFSETS = 9, /* int64 [M+1] first word of block b inside a row of SIGN_BITS            */
+    COMPAMS_BUF_SCALES = 10,      /* float  [n, M]   Block-Sign scales ||x_B||_1 / d_B                           */
+    COMPAMS_BUF_STATUS = 11       /* uint32 [1]      device status word (0 = clean)                              */
+};
+
+/* Kernel identifiers for compams_get_kernel_time. */
+enum compams_kernel {
+    COMPAMS_K_DENSE_MEAN_AMSGRAD = 0, /* k = d: mean over workers fused with the AMSGrad update              */
+    COMPAMS_K_BS_SWEEP = 1,           /* Block-Sign: EF add, block |x| partial sums, sign pack                */
+    COMPAMS_K_BS_APPLY = 2,           /* Block-Sign: segmented average over workers fused with AMSGrad        */
+    COMPAMS_K_BS_MATERIALIZE = 3,     /* Block-Sign: turn the stored x into e when E is read                  */
+    COMPAMS_K_TOPK_SWEEP = 4,         /* Top-k: EF add, x written to E, first radix histogram                 */
+    COMPAMS_K_TOPK_HIST = 5,          /* Top-k: later radix histogram passes                                  */
+    COMPAMS_K_TOPK_FIND = 6,          /* Top-k: locate the threshold bin of a pass                            */
+    COMPAMS_K_TOPK_COLLECT = 7,       /* Top-k: emit (index, value), zero kept e, count threshold ties        */
+    COMPAMS_K_TOPK_TIES = 8,          /* Top-k: take the lowest-index ties at the threshold                   */
+    COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: sparse scatter-accumulate into the averaged gradient          */
+    COMPAMS_K_AMSGRAD = 10,           /* Top-k: AMSGrad update from the accumulated average                   */
+    COMPAMS_K_TOPK_SMALL = 11,        /* Top-k: whole small blocks selected inside shared memory              */
+    COMPAMS_K_COUNT = 12
+};
+
+/*
+ * compams_create - build the optimizer state (Algorithm 2, "Initialize": e_{1,i} = 0,
+ * m_0 = v_0 = vhat_0 = 0).
+ *
+ *   out            host; receives the handle. Untouched on failure.
+ *   n              number of simulated workers, 1 <= n <= 65535.
+ *   d              number of parameters, 1 <= d < 2^31.
+ *   block_offsets  host; num_blocks + 1 entries, [0] = 0, strictly increasing, last = d. Copied.
+ *   num_blocks     M >= 1. The compressor acts on each block separately (Section 3.1). With one
+ *                  block Top-k is taken over the whole vector; with one block per tensor it is
+ *                  layer-wise.
+ *   compressor     COMPAMS_TOPK or COMPAMS_BLOCKSIGN.
+ *   k_ratio        Top-k only, in (0, 1]: block b keeps k_b = max(1, min(d_b, floor(k_ratio * d_b)))
+ *                  coordinates (Section 5.1 uses 0.01). If every k_b equals d_b the compressor is
+ *                  the identity (q = 0 in Assumption 1): the step is then full-precision
+ *                  distributed AMSGrad, e stays 0 and no (index, value) message is produced.
+ *                  Ignored for Block-Sign.
+ *   lr, beta1, beta2, eps   AMSGrad hyper-parameters (Algorithm 1); eps is added under the root.
+ *
+ * Allocates, on the current CUDA device, E [n, d], m, v, vhat, gbar [d], the message buffers and
+ * scratch, all owned by the handle and zero-initialised. Synchronises the device once.
+ * Errors: INVALID_ARG for any violated range above; ALLOC; CUDA.
+ */
+int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* block_offsets, int32_t num_blocks,
+                   int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps);
+
+/*
+ * compams_step - one iteration of Algorithm 2 (lines 7-8 for every worker, lines 12-16 for the
+ * server), enqueued on the handle's stream.
+ *
+ *   grads   device; [n, d] fp32, packed row-major (row i = g_{t,i}, row stride d), 4-byte aligned.
+ *           Read only; must stay valid and unchanged until the enqueued work has run.
+ *   theta   device; [d] fp32 parameters theta_t, overwritten with theta_{t+1}. 16-byte aligned.
+ *
+ * After the step: BUF_E holds e_{t+1}, BUF_GBAR holds gbar_t, BUF_M/V/VHAT the moments, and
+ * the message buffers hold what each worker would have sent: for Top-k the k_b (index, value)
+ * pairs of every (worker, block) - in no particular order inside a segment, ties at the
+ * threshold magnitude resolved towards the lower index - and for Block-Sign one sign bit per
+ * coordinate plus one scale per (worker, block). sign(x) follows the IEEE sign bit (+0 -> +,
+ * -0 -> -), so every coordinate of a block contributes exactly +-scale.
+ * Errors: INVALID_ARG (null or misaligned pointer), CUDA (launch failure).
+ */
+int compams_step(compams_handle h, const float* grads, float* theta);
+
+/*
+ * compams_step_host - the same iteration for callers whose tensors live in HOST memory
+ * (Algorithm 2's "send g~ to the server / receive theta" endpoints on a machine where the
+ * gradients are produced off-GPU).
+ *
+ *   grads_host  host; [n, d] fp32 packed. Copied to a device staging buffer owned by the handle.
+ *   theta_host  host; [d] fp32; copied in, updated, copied back.
+ *
+ * Enqueues copy-in, the step and copy-out on the handle's stream and then SYNCHRONISES the
+ * stream, so on return theta_host holds theta_{t+1}. Pinned host memory makes the copies faster
+ * but is not required. The staging buffers are allocated on first use.
+ */
+int compams_step_host(compams_handle h, const float* grads_host, float* theta_host);
+
+/* compams_destroy - free everything the handle owns (synchronises its stream first).
+ * A null handle is a no-op. */
+int compams_destroy(compams_handle h);
+
+/* compams_set_stream - use `cuda_stream` (a cudaStream_t passed as void*, null = default stream)
+ * for all later work of this handle. The caller orders earlier work against the new stream. */
+int compams_set_stream(compams_handle h, void* cuda_stream);
+
+/* compams_set_lr - learning rate eta_t for the following steps (Algorithm 2 allows it to vary
+ * with t; Section 5.2 divides it by 10 at fixed epochs). */
+int compams_set_lr(compams_handle h, float lr);
+
+/*
+ * compams_get_buffer - device pointer and element count of one of the handle's buffers.
+ *
+ *   which     a compams_buffer value.
+ *   dev_ptr   host; receives the DEVICE pointer (read-only for the caller).
+ *   count     host; receives the number of elements (0 if the buffer does not exist for this
+ *             compressor, in which case *dev_ptr is null).
+ *
+ * The contents are those of the last enqueued step once the stream has reached that point;
+ * they stay valid until the next compams_step / compams_destroy. Asking for BUF_E of a
+ * Block-Sign handle enqueues one extra kernel that turns the stored corrected gradient x into
+ * the residual e = x - g~ in place (the step itself defers that subtraction to the next
+ * iteration's sweep; values are identical either way).
+ *
+ * SIGN_BITS layout: row i has W words; block b starts at word SIGN_WORD_OFFSETS[b]; bit (r % 32)
+ * of word SIGN_WORD_OFFSETS[b] + r / 32 is the sign bit of x at coordinate block_offsets[b] + r;
+ * unused high bits of a block's last word are 0.
+ */
+int compams_get_buffer(compams_handle h, int32_t which, void** dev_ptr, int64_t* count);
+
+/* compams_check_status - synchronise the handle's stream, read the device status word and any
+ * pending CUDA error. Returns OK, ERR_CUDA or ERR_DEVICE_STATUS; *status_word (host, may be null)
+ * receives the raw word (bit 0: a Top-k segment emitted a wrong number of entries). */
+int compams_check_status(compams_handle h, uint32_t* status_word);
+
+/*
+ * Per-kernel timing with CUDA events on the handle's stream.
+ *   compams_set_profiling(h, mask): bit k of mask enables an event pair around every launch of
+ *     kernel k (compams_kernel) in later steps; 0 disables. Timing state is reset.
+ *   compams_get_kernel_time(h, k, &ms, &launches): synchronises the stream and returns the summed
+ *     device time and launch count of kernel k since profiling was enabled.
+ * At most 4096 launches are recorded between two resets; later ones are not timed.
+ */
+int compams_set_profiling(compams_handle h, uint32_t kernel_mask);
+int compams_get_kernel_time(compams_handle h, int32_t kernel, double* total_ms, int64_t* launches);
+
+/* Number of kernel launches the handle has enqueued since creation (all kernels, all steps). */
+int64_t compams_launch_count(compams_handle h);
+
+/* Static strings (never null). */
+const char* compams_error_string(int status);
+const char* compams_kernel_name(int32_t kernel);
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char* compams_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMPAMS_H */

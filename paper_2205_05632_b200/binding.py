@@ -1,0 +1,220 @@
+"""ctypes binding of the COMP-AMS C ABI (include/compams.h).
+
+Argument marshalling only: every step of the optimizer iteration runs inside the CUDA library.
+PyTorch supplies device memory and the CUDA stream. If the compiled library is missing the
+first call raises CompAMSError; there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+TOPK = 0
+BLOCKSIGN = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_NAME = "libcompams.so"
+
+BUFFERS = {
+    "E": 0, "m": 1, "v": 2, "vhat": 3, "gbar": 4, "topk_idx": 5, "topk_val": 6, "topk_seg_offsets": 7,
+    "sign_bits": 8, "sign_word_offsets": 9, "scales": 10, "status": 11,
+}
+_BUFFER_DTYPES = {
+    "E": torch.float32, "m": torch.float32, "v": torch.float32, "vhat": torch.float32, "gbar": torch.float32,
+    "topk_idx": torch.int32, "topk_val": torch.float32, "topk_seg_offsets": torch.int64,
+    "sign_bits": torch.int32, "sign_word_offsets": torch.int64, "scales": torch.float32, "status": torch.int32,
+}
+_TYPESTR = {torch.float32: "<f4", torch.int32: "<i4", torch.int64: "<i8"}
+
+KERNELS = {
+    "dense_mean_amsgrad": 0, "bs_sweep": 1, "bs_apply": 2, "bs_materialize": 3, "topk_sweep": 4, "topk_hist": 5,
+    "topk_find": 6, "topk_collect": 7, "topk_ties": 8, "topk_scatter": 9, "amsgrad": 10, "topk_small": 11,
+}
+
+
+class CompAMSError(RuntimeError):
+    pass
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, _LIB_NAME)
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libcompams.so (built in-tree by paper_2205_05632_b200.build) and declare its symbols."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise CompAMSError(
+            "CUDA library %s not found: build it with `python -m paper_2205_05632_b200.build` "
+            "(there is no CPU fallback)" % path)
+    L = ctypes.CDLL(path)
+    c = ctypes
+    H = c.c_void_p
+    L.compams_create.restype = c.c_int
+    L.compams_create.argtypes = [c.POINTER(H), c.c_int32, c.c_int64, c.POINTER(c.c_int64), c.c_int32, c.c_int32,
+                                 c.c_double, c.c_float, c.c_float, c.c_float, c.c_float]
+    L.compams_step.restype = c.c_int
+    L.compams_step.argtypes = [H, c.c_void_p, c.c_void_p]
+    L.compams_step_host.restype = c.c_int
+    L.compams_step_host.argtypes = [H, c.c_void_p, c.c_void_p]
+    L.compams_destroy.restype = c.c_int
+    L.compams_destroy.argtypes = [H]
+    L.compams_set_stream.restype = c.c_int
+    L.compams_set_stream.argtypes = [H, c.c_void_p]
+    L.compams_set_lr.restype = c.c_int
+    L.compams_set_lr.argtypes = [H, c.c_float]
+    L.compams_get_buffer.restype = c.c_int
+    L.compams_get_buffer.argtypes = [H, c.c_int32, c.POINTER(c.c_void_p), c.POINTER(c.c_int64)]
+    L.compams_check_status.restype = c.c_int
+    L.compams_check_status.argtypes = [H, c.POINTER(c.c_uint32)]
+    L.compams_set_profiling.restype = c.c_int
+    L.compams_set_profiling.argtypes = [H, c.c_uint32]
+    L.compams_get_kernel_time.restype = c.c_int
+    L.compams_get_kernel_time.argtypes = [H, c.c_int32, c.POINTER(c.c_double), c.POINTER(c.c_int64)]
+    L.compams_launch_count.restype = c.c_int64
+    L.compams_launch_count.argtypes = [H]
+    L.compams_error_string.restype = c.c_char_p
+    L.compams_error_string.argtypes = [c.c_int]
+    L.compams_kernel_name.restype = c.c_char_p
+    L.compams_kernel_name.argtypes = [c.c_int32]
+    L.compams_last_cuda_error.restype = c.c_char_p
+    L.compams_last_cuda_error.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        L = load_library()
+        msg = L.compams_error_string(rc).decode()
+        cuda = L.compams_last_cuda_error().decode()
+        raise CompAMSError("%s failed: %s (%d)%s" % (what, msg, rc, (" [" + cuda + "]") if cuda else ""))
+
+
+class _DeviceView:
+    """Exposes a raw device pointer to torch through the CUDA array interface."""
+
+    def __init__(self, ptr: int, count: int, dtype: torch.dtype, owner):
+        self.__cuda_array_interface__ = {
+            "shape": (count,), "typestr": _TYPESTR[dtype], "data": (ptr, False), "version": 2, "strides": None,
+        }
+        self._owner = owner
+
+
+class CompAMS:
+    """One COMP-AMS optimizer (Algorithm 2) on the current CUDA device.
+
+    `step(grads, theta)` takes device tensors; `step_host(grads, theta)` takes host tensors and
+    includes the transfers. `buffer(name)` returns a torch view of a library-owned device buffer.
+    """
+
+    def __init__(self, n: int, d: int, block_offsets: Sequence[int], compressor: int, k_ratio: float = 1.0,
+                 lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                 stream: Optional[torch.cuda.Stream] = None):
+        self._L = load_library()
+        self.n, self.d = int(n), int(d)
+        offs = np.ascontiguousarray(block_offsets, dtype=np.int64)
+        self.M = int(offs.size - 1)
+        self.compressor = int(compressor)
+        self._h = ctypes.c_void_p()
+        rc = self._L.compams_create(ctypes.byref(self._h), self.n, self.d,
+                                    offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), self.M, self.compressor,
+                                    float(k_ratio), float(lr), float(beta1), float(beta2), float(eps))
+        if rc != 0:
+            self._h = ctypes.c_void_p()
+        _check(rc, "compams_create")
+        self.set_stream(stream if stream is not None else torch.cuda.current_stream())
+
+    # -- calls ---------------------------------------------------------------------------------
+    def set_stream(self, stream: torch.cuda.Stream) -> None:
+        _check(self._L.compams_set_stream(self._h, ctypes.c_void_p(stream.cuda_stream)), "compams_set_stream")
+
+    def set_lr(self, lr: float) -> None:
+        _check(self._L.compams_set_lr(self._h, float(lr)), "compams_set_lr")
+
+    def step(self, grads: torch.Tensor, theta: torch.Tensor) -> None:
+        if not (grads.is_cuda and theta.is_cuda):
+            raise CompAMSError("step() takes CUDA tensors; use step_host() for host tensors")
+        if grads.dtype != torch.float32 or theta.dtype != torch.float32:
+            raise CompAMSError("grads and theta must be float32")
+        if tuple(grads.shape) != (self.n, self.d) or not grads.is_contiguous():
+            raise CompAMSError("grads must be a contiguous [n, d] tensor")
+        if tuple(theta.shape) != (self.d,) or not theta.is_contiguous():
+            raise CompAMSError("theta must be a contiguous [d] tensor")
+        _check(self._L.compams_step(self._h, ctypes.c_void_p(grads.data_ptr()), ctypes.c_void_p(theta.data_ptr())),
+               "compams_step")
+
+    def step_host(self, grads: torch.Tensor, theta: torch.Tensor) -> None:
+        if grads.is_cuda or theta.is_cuda:
+            raise CompAMSError("step_host() takes host tensors")
+        if grads.dtype != torch.float32 or theta.dtype != torch.float32:
+            raise CompAMSError("grads and theta must be float32")
+        if tuple(grads.shape) != (self.n, self.d) or not grads.is_contiguous():
+            raise CompAMSError("grads must be a contiguous [n, d] tensor")
+        if tuple(theta.shape) != (self.d,) or not theta.is_contiguous():
+            raise CompAMSError("theta must be a contiguous [d] tensor")
+        _check(self._L.compams_step_host(self._h, ctypes.c_void_p(grads.data_ptr()),
+                                         ctypes.c_void_p(theta.data_ptr())), "compams_step_host")
+
+    def buffer(self, name: str) -> torch.Tensor:
+        """Torch view of a library-owned device buffer (valid until the next step / close)."""
+        which = BUFFERS[name]
+        ptr = ctypes.c_void_p()
+        cnt = ctypes.c_int64()
+        _check(self._L.compams_get_buffer(self._h, which, ctypes.byref(ptr), ctypes.byref(cnt)),
+               "compams_get_buffer")
+        dt = _BUFFER_DTYPES[name]
+        if cnt.value == 0 or not ptr.value:
+            return torch.empty(0, dtype=dt, device="cuda")
+        t = torch.as_tensor(_DeviceView(ptr.value, cnt.value, dt, self), device="cuda")
+        if name == "E":
+            return t.view(self.n, self.d)
+        if name in ("topk_idx", "topk_val", "sign_bits"):
+            return t.view(self.n, -1)
+        if name == "scales":
+            return t.view(self.n, self.M)
+        return t
+
+    def check_status(self) -> int:
+        word = ctypes.c_uint32(0)
+        rc = self._L.compams_check_status(self._h, ctypes.byref(word))
+        _check(rc, "compams_check_status (status word 0x%x)" % word.value)
+        return int(word.value)
+
+    def set_profiling(self, kernels: Sequence[str]) -> None:
+        mask = 0
+        for k in kernels:
+            mask |= 1 << KERNELS[k]
+        _check(self._L.compams_set_profiling(self._h, mask), "compams_set_profiling")
+
+    def kernel_time(self, kernel: str):
+        """(total device milliseconds, launches) of one kernel since set_profiling()."""
+        ms = ctypes.c_double(0.0)
+        cnt = ctypes.c_int64(0)
+        _check(self._L.compams_get_kernel_time(self._h, KERNELS[kernel], ctypes.byref(ms), ctypes.byref(cnt)),
+               "compams_get_kernel_time")
+        return ms.value, int(cnt.value)
+
+    def launch_count(self) -> int:
+        return int(self._L.compams_launch_count(self._h))
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._L.compams_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
