@@ -1,0 +1,439 @@
+// C ABI of the COMP-AMS library (see include/compams.h): argument checks, state allocation,
+// the per-step launch sequence and the inspection calls.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "context.h"
+
+using namespace compams;
+
+namespace {
+
+thread_local std::string g_last_cuda_error;
+
+int cuda_fail(cudaError_t e, const char* what) {
+    g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return COMPAMS_ERR_CUDA;
+}
+
+#define CU(call)                                          \
+    do {                                                  \
+        cudaError_t _e = (call);                          \
+        if (_e != cudaSuccess) return cuda_fail(_e, #call); \
+    } while (0)
+
+template <typename T>
+int dev_alloc(compams_context* c, T** out, size_t count, bool zero = true) {
+    *out = nullptr;
+    if (count == 0) count = 1;
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, count * sizeof(T));
+    if (e != cudaSuccess) {
+        g_last_cuda_error = std::string("cudaMalloc: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return COMPAMS_ERR_ALLOC;
+    }
+    c->owned.push_back(p);
+    if (zero) CU(cudaMemsetAsync(p, 0, count * sizeof(T), c->stream));
+    *out = (T*)p;
+    return COMPAMS_OK;
+}
+
+template <typename T>
+int dev_upload(compams_context* c, T** out, const std::vector<T>& host) {
+    int rc = dev_alloc(c, out, host.size(), false);
+    if (rc) return rc;
+    if (!host.empty()) CU(cudaMemcpy(*out, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice));
+    return COMPAMS_OK;
+}
+
+#define RC(call)              \
+    do {                      \
+        int _rc = (call);     \
+        if (_rc) return _rc;  \
+    } while (0)
+
+int64_t kept_per_block(double k_ratio, int64_t d_b) {
+    int64_t k = (int64_t)std::floor(k_ratio * (double)d_b);
+    if (k < 1) k = 1;
+    if (k > d_b) k = d_b;
+    return k;
+}
+
+// Cuts the listed blocks into tiles of kTile coordinates and uploads the tables.
+int build_tiles(compams_context* c, const std::vector<int32_t>& blocks) {
+    std::vector<int32_t> tile_blk, tile_r0, tile_seg, seg_tile0;
+    seg_tile0.push_back(0);
+    for (size_t s = 0; s < blocks.size(); ++s) {
+        const int32_t b = blocks[s];
+        const int64_t len = c->off[b + 1] - c->off[b];
+        for (int64_t r0 = 0; r0 < len; r0 += kTile) {
+            tile_blk.push_back(b);
+            tile_r0.push_back((int32_t)r0);
+            tile_seg.push_back((int32_t)s);
+        }
+        if (tile_blk.size() > (size_t)0x7fffffff) return COMPAMS_ERR_INVALID_ARG;
+        seg_tile0.push_back((int32_t)tile_blk.size());
+    }
+    int32_t *d_blk, *d_r0, *d_seg, *d_t0;
+    RC(dev_upload(c, &d_blk, tile_blk));
+    RC(dev_upload(c, &d_r0, tile_r0));
+    RC(dev_upload(c, &d_seg, tile_seg));
+    RC(dev_upload(c, &d_t0, seg_tile0));
+    c->tab.ntiles = (int32_t)tile_blk.size();
+    c->tab.tile_blk = d_blk;
+    c->tab.tile_r0 = d_r0;
+    c->tab.tile_seg = d_seg;
+    c->tab.seg_tile0 = d_t0;
+    c->tab.nseg = (int32_t)blocks.size();
+    return COMPAMS_OK;
+}
+
+int init_context(compams_context* c, const int64_t* block_offsets) {
+    CU(cudaGetDevice(&c->device));
+    CU(cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device));
+    const int32_t n = c->n, M = c->M;
+    const int64_t d = c->d;
+    c->off.assign(block_offsets, block_offsets + M + 1);
+    c->tab.n = n;
+    c->tab.d = d;
+    c->tab.M = M;
+    RC(dev_upload(c, &c->d_off, c->off));
+    c->tab.off = c->d_off;
+
+    RC(dev_alloc(c, &c->m, (size_t)d));
+    RC(dev_alloc(c, &c->v, (size_t)d));
+    RC(dev_alloc(c, &c->vhat, (size_t)d));
+    RC(dev_alloc(c, &c->gbar, (size_t)d));
+    RC(dev_alloc(c, &c->status, 1));
+
+    if (c->compressor == COMPAMS_TOPK) {
+        c->seg_off.assign((size_t)M + 1, 0);
+        bool identity = true;
+        for (int32_t b = 0; b < M; ++b) {
+            const int64_t db = c->off[b + 1] - c->off[b];
+            const int64_t kb = kept_per_block(c->k_ratio, db);
+            identity = identity && (kb == db);
+            c->seg_off[(size_t)b + 1] = c->seg_off[(size_t)b] + kb;
+        }
+        c->identity = identity;
+        c->K = identity ? 0 : c->seg_off[(size_t)M];
+    }
+
+    if (c->compressor == COMPAMS_TOPK && c->identity) {
+        // full-precision distributed AMSGrad: e is identically zero, kept only so that BUF_E can be read
+        RC(dev_alloc(c, &c->E, (size_t)n * (size_t)d));
+    } else if (c->compressor == COMPAMS_TOPK) {
+        RC(dev_alloc(c, &c->E, (size_t)n * (size_t)d));
+        RC(dev_upload(c, &c->d_seg_off, c->seg_off));
+        std::vector<int32_t> small, large;
+        for (int32_t b = 0; b < M; ++b) ((c->off[b + 1] - c->off[b] <= kSmallMax) ? small : large).push_back(b);
+        RC(build_tiles(c, large));
+        TopkBuffers& t = c->tk;
+        t.E = c->E;
+        t.K = c->K;
+        t.seg_off = c->d_seg_off;
+        int32_t* d_small;
+        RC(dev_upload(c, &d_small, small));
+        t.small_blk = d_small;
+        t.nsmall = (int32_t)small.size();
+        RC(dev_alloc(c, &t.idx, (size_t)n * (size_t)c->K));
+        RC(dev_alloc(c, &t.val, (size_t)n * (size_t)c->K));
+        RC(dev_alloc(c, &t.hist, (size_t)n * (size_t)c->tab.nseg * kBins1));
+        RC(dev_alloc(c, &t.seg, (size_t)n * (size_t)c->tab.nseg));
+        RC(dev_alloc(c, &t.tile_ties, (size_t)n * (size_t)c->tab.ntiles));
+        RC(dev_alloc(c, &t.acc, (size_t)d));
+        t.status = c->status;
+        t.gbar = c->gbar;
+        t.m = c->m;
+        t.v = c->v;
+        t.vhat = c->vhat;
+    } else {
+        RC(dev_alloc(c, &c->E, (size_t)n * (size_t)d));
+        std::vector<int32_t> all((size_t)M);
+        for (int32_t b = 0; b < M; ++b) all[(size_t)b] = b;
+        RC(build_tiles(c, all));
+        std::vector<int64_t> word_off((size_t)M + 1, 0);
+        for (int32_t b = 0; b < M; ++b)
+            word_off[(size_t)b + 1] = word_off[(size_t)b] + (c->off[b + 1] - c->off[b] + 31) / 32;
+        c->W = word_off[(size_t)M];
+        RC(dev_upload(c, &c->d_word_off, word_off));
+        BsBuffers& s = c->bs;
+        s.E = c->E;
+        s.word_off = c->d_word_off;
+        s.W = c->W;
+        RC(dev_alloc(c, &s.bits, (size_t)n * (size_t)c->W));
+        RC(dev_alloc(c, &c->scales[0], (size_t)n * (size_t)M));
+        RC(dev_alloc(c, &c->scales[1], (size_t)n * (size_t)M));
+        RC(dev_alloc(c, &s.tile_sum, (size_t)n * (size_t)c->tab.ntiles));
+        RC(dev_alloc(c, &s.ticket, (size_t)n * (size_t)M));
+        s.gbar = c->gbar;
+        s.m = c->m;
+        s.v = c->v;
+        s.vhat = c->vhat;
+    }
+    CU(cudaDeviceSynchronize());
+    return COMPAMS_OK;
+}
+
+void free_context(compams_context* c) {
+    for (void* p : c->owned) cudaFree(p);
+    c->owned.clear();
+    if (c->stage_grads) cudaFree(c->stage_grads);
+    if (c->stage_theta) cudaFree(c->stage_theta);
+    for (cudaEvent_t e : c->ev_start) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->ev_stop) cudaEventDestroy(e);
+    delete c;
+}
+
+// Runs one launcher, optionally bracketed by an event pair for per-kernel timing.
+template <typename F>
+int run_kernel(compams_context* c, int kernel, F&& launch) {
+    const bool timed = (c->prof_mask >> kernel) & 1u;
+    int slot = -1;
+    if (timed && c->prof_used < kMaxTimed) {
+        slot = c->prof_used++;
+        if ((size_t)slot >= c->ev_start.size()) {
+            cudaEvent_t a, b;
+            CU(cudaEventCreate(&a));
+            CU(cudaEventCreate(&b));
+            c->ev_start.push_back(a);
+            c->ev_stop.push_back(b);
+            c->ev_kernel.push_back(kernel);
+        }
+        c->ev_kernel[(size_t)slot] = kernel;
+        CU(cudaEventRecord(c->ev_start[(size_t)slot], c->stream));
+    }
+    cudaError_t e = launch();
+    if (e != cudaSuccess) return cuda_fail(e, compams_kernel_name(kernel));
+    ++c->launches;
+    if (slot >= 0) CU(cudaEventRecord(c->ev_stop[(size_t)slot], c->stream));
+    return COMPAMS_OK;
+}
+
+int step_device(compams_context* c, const float* grads, float* theta) {
+    if (c->compressor == COMPAMS_TOPK && c->identity) {
+        return run_kernel(c, COMPAMS_K_DENSE_MEAN_AMSGRAD, [&] { return launch_dense_mean_amsgrad(c, grads, theta); });
+    }
+    if (c->compressor == COMPAMS_BLOCKSIGN) {
+        c->scales_cur ^= 1;
+        RC(run_kernel(c, COMPAMS_K_BS_SWEEP, [&] { return launch_bs_sweep(c, grads); }));
+        c->e_is_x = true;
+        RC(run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); }));
+        return COMPAMS_OK;
+    }
+    if (c->tk.nsmall > 0) RC(run_kernel(c, COMPAMS_K_TOPK_SMALL, [&] { return launch_topk_small(c, grads); }));
+    if (c->tab.ntiles > 0) {
+        RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 1); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 2); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 2); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 3); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 3); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_COLLECT, [&] { return launch_topk_collect(c); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_TIES, [&] { return launch_topk_ties(c); }));
+    }
+    RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c); }));
+    RC(run_kernel(c, COMPAMS_K_AMSGRAD, [&] { return launch_amsgrad(c, theta); }));
+    return COMPAMS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* block_offsets, int32_t num_blocks,
+                   int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps) {
+    if (!out || !block_offsets) return COMPAMS_ERR_INVALID_ARG;
+    if (n < 1 || n > 65535 || d < 1 || d >= ((int64_t)1 << 31) || num_blocks < 1 || (int64_t)num_blocks > d)
+        return COMPAMS_ERR_INVALID_ARG;
+    if (compressor != COMPAMS_TOPK && compressor != COMPAMS_BLOCKSIGN) return COMPAMS_ERR_INVALID_ARG;
+    if (compressor == COMPAMS_TOPK && !(k_ratio > 0.0 && k_ratio <= 1.0)) return COMPAMS_ERR_INVALID_ARG;
+    if (!(lr == lr) || !(beta1 == beta1) || !(beta2 == beta2) || !(eps == eps)) return COMPAMS_ERR_INVALID_ARG;
+    if (block_offsets[0] != 0 || block_offsets[num_blocks] != d) return COMPAMS_ERR_INVALID_ARG;
+    for (int32_t b = 0; b < num_blocks; ++b)
+        if (block_offsets[b + 1] <= block_offsets[b]) return COMPAMS_ERR_INVALID_ARG;
+
+    compams_context* c = new (std::nothrow) compams_context();
+    if (!c) return COMPAMS_ERR_ALLOC;
+    c->n = n;
+    c->d = d;
+    c->M = num_blocks;
+    c->compressor = compressor;
+    c->k_ratio = (compressor == COMPAMS_TOPK) ? k_ratio : 1.0;
+    c->hp.lr = lr;
+    c->hp.beta1 = beta1;
+    c->hp.beta2 = beta2;
+    c->hp.omb1 = 1.0f - beta1;
+    c->hp.omb2 = 1.0f - beta2;
+    c->hp.eps = eps;
+    c->hp.nf = (float)n;
+    int rc;
+    try {
+        rc = init_context(c, block_offsets);
+    } catch (const std::bad_alloc&) {
+        rc = COMPAMS_ERR_ALLOC;
+    }
+    if (rc) {
+        free_context(c);
+        return rc;
+    }
+    *out = c;
+    return COMPAMS_OK;
+}
+
+int compams_step(compams_handle c, const float* grads, float* theta) {
+    if (!c || !grads || !theta) return COMPAMS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(grads) & 3u) || (reinterpret_cast<uintptr_t>(theta) & 15u))
+        return COMPAMS_ERR_INVALID_ARG;
+    try {
+        return step_device(c, grads, theta);
+    } catch (const std::bad_alloc&) {
+        return COMPAMS_ERR_ALLOC;
+    }
+}
+
+int compams_step_host(compams_handle c, const float* grads_host, float* theta_host) {
+    if (!c || !grads_host || !theta_host) return COMPAMS_ERR_INVALID_ARG;
+    const size_t gbytes = (size_t)c->n * (size_t)c->d * sizeof(float);
+    const size_t tbytes = (size_t)c->d * sizeof(float);
+    if (!c->stage_grads) {
+        cudaError_t e = cudaMalloc((void**)&c->stage_grads, gbytes);
+        if (e != cudaSuccess) {
+            c->stage_grads = nullptr;
+            cudaGetLastError();
+            return COMPAMS_ERR_ALLOC;
+        }
+        e = cudaMalloc((void**)&c->stage_theta, tbytes);
+        if (e != cudaSuccess) {
+            c->stage_theta = nullptr;
+            cudaGetLastError();
+            return COMPAMS_ERR_ALLOC;
+        }
+    }
+    CU(cudaMemcpyAsync(c->stage_grads, grads_host, gbytes, cudaMemcpyHostToDevice, c->stream));
+    CU(cudaMemcpyAsync(c->stage_theta, theta_host, tbytes, cudaMemcpyHostToDevice, c->stream));
+    int rc;
+    try {
+        rc = step_device(c, c->stage_grads, c->stage_theta);
+    } catch (const std::bad_alloc&) {
+        rc = COMPAMS_ERR_ALLOC;
+    }
+    if (rc) return rc;
+    CU(cudaMemcpyAsync(theta_host, c->stage_theta, tbytes, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    return COMPAMS_OK;
+}
+
+int compams_destroy(compams_handle c) {
+    if (!c) return COMPAMS_OK;
+    cudaStreamSynchronize(c->stream);
+    free_context(c);
+    return COMPAMS_OK;
+}
+
+int compams_set_stream(compams_handle c, void* cuda_stream) {
+    if (!c) return COMPAMS_ERR_INVALID_ARG;
+    c->stream = (cudaStream_t)cuda_stream;
+    return COMPAMS_OK;
+}
+
+int compams_set_lr(compams_handle c, float lr) {
+    if (!c || !(lr == lr)) return COMPAMS_ERR_INVALID_ARG;
+    c->hp.lr = lr;
+    return COMPAMS_OK;
+}
+
+int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t* count) {
+    if (!c || !dev_ptr || !count) return COMPAMS_ERR_INVALID_ARG;
+    void* p = nullptr;
+    int64_t cnt = 0;
+    const bool topk = c->compressor == COMPAMS_TOPK && !c->identity;
+    const bool sign = c->compressor == COMPAMS_BLOCKSIGN;
+    switch (which) {
+        case COMPAMS_BUF_E:
+            if (sign && c->e_is_x) {
+                RC(run_kernel(c, COMPAMS_K_BS_MATERIALIZE, [&] { return launch_bs_materialize(c); }));
+                c->e_is_x = false;
+            }
+            p = c->E;
+            cnt = (int64_t)c->n * c->d;
+            break;
+        case COMPAMS_BUF_M: p = c->m; cnt = c->d; break;
+        case COMPAMS_BUF_V: p = c->v; cnt = c->d; break;
+        case COMPAMS_BUF_VHAT: p = c->vhat; cnt = c->d; break;
+        case COMPAMS_BUF_GBAR: p = c->gbar; cnt = c->d; break;
+        case COMPAMS_BUF_TOPK_IDX: if (topk) { p = c->tk.idx; cnt = (int64_t)c->n * c->K; } break;
+        case COMPAMS_BUF_TOPK_VAL: if (topk) { p = c->tk.val; cnt = (int64_t)c->n * c->K; } break;
+        case COMPAMS_BUF_TOPK_SEG_OFFSETS: if (topk) { p = c->d_seg_off; cnt = c->M + 1; } break;
+        case COMPAMS_BUF_SIGN_BITS: if (sign) { p = c->bs.bits; cnt = (int64_t)c->n * c->W; } break;
+        case COMPAMS_BUF_SIGN_WORD_OFFSETS: if (sign) { p = c->d_word_off; cnt = c->M + 1; } break;
+        case COMPAMS_BUF_SCALES: if (sign) { p = c->scales[c->scales_cur]; cnt = (int64_t)c->n * c->M; } break;
+        case COMPAMS_BUF_STATUS: p = c->status; cnt = 1; break;
+        default: return COMPAMS_ERR_INVALID_ARG;
+    }
+    *dev_ptr = p;
+    *count = cnt;
+    return COMPAMS_OK;
+}
+
+int compams_check_status(compams_handle c, uint32_t* status_word) {
+    if (!c) return COMPAMS_ERR_INVALID_ARG;
+    CU(cudaStreamSynchronize(c->stream));
+    uint32_t w = 0;
+    CU(cudaMemcpy(&w, c->status, sizeof w, cudaMemcpyDeviceToHost));
+    if (status_word) *status_word = w;
+    return w ? COMPAMS_ERR_DEVICE_STATUS : COMPAMS_OK;
+}
+
+int compams_set_profiling(compams_handle c, uint32_t kernel_mask) {
+    if (!c) return COMPAMS_ERR_INVALID_ARG;
+    CU(cudaStreamSynchronize(c->stream));
+    c->prof_mask = kernel_mask;
+    c->prof_used = 0;
+    return COMPAMS_OK;
+}
+
+int compams_get_kernel_time(compams_handle c, int32_t kernel, double* total_ms, int64_t* launches) {
+    if (!c || !total_ms || !launches || kernel < 0 || kernel >= COMPAMS_K_COUNT) return COMPAMS_ERR_INVALID_ARG;
+    CU(cudaStreamSynchronize(c->stream));
+    double ms = 0.0;
+    int64_t cnt = 0;
+    for (int s = 0; s < c->prof_used; ++s) {
+        if (c->ev_kernel[(size_t)s] != kernel) continue;
+        float t = 0.0f;
+        CU(cudaEventElapsedTime(&t, c->ev_start[(size_t)s], c->ev_stop[(size_t)s]));
+        ms += (double)t;
+        ++cnt;
+    }
+    *total_ms = ms;
+    *launches = cnt;
+    return COMPAMS_OK;
+}
+
+int64_t compams_launch_count(compams_handle c) { return c ? c->launches : 0; }
+
+const char* compams_error_string(int status) {
+    switch (status) {
+        case COMPAMS_OK: return "ok";
+        case COMPAMS_ERR_INVALID_ARG: return "invalid argument";
+        case COMPAMS_ERR_ALLOC: return "allocation failed";
+        case COMPAMS_ERR_CUDA: return "CUDA runtime error";
+        case COMPAMS_ERR_DEVICE_STATUS: return "device status word is set";
+        default: return "unknown status";
+    }
+}
+
+const char* compams_kernel_name(int32_t kernel) {
+    static const char* names[COMPAMS_K_COUNT] = {
+        "dense_mean_amsgrad", "bs_sweep", "bs_apply", "bs_materialize", "topk_sweep", "topk_hist",
+        "topk_find", "topk_collect", "topk_ties", "topk_scatter", "amsgrad", "topk_small"};
+    return (kernel >= 0 && kernel < COMPAMS_K_COUNT) ? names[kernel] : "unknown";
+}
+
+const char* compams_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,129 @@
+// Device helpers shared by the COMP-AMS kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace compams {
+
+constexpr int kThreads = 256;          // threads per CTA of every tiled kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kTile = 8192;            // coordinates per tile: 8 warps x 8 iterations x 32 lanes x 4
+constexpr int kWarpSpan = kTile / kWarps;  // 1024 consecutive coordinates per warp
+constexpr int kIters = kWarpSpan / 128;    // 8 iterations of one float4 per lane
+
+// AMSGrad hyper-parameters as the fp32 numbers every kernel uses (Algorithm 1).
+struct HyperParams {
+    float lr, beta1, beta2, omb1, omb2, eps, nf;  // omb = 1 - beta (fp32), nf = (float)n
+};
+
+// One AMSGrad coordinate update (Algorithm 2, lines 13-16). Every operation is a separately
+// rounded fp32 operation: no fused multiply-add, IEEE square root and division.
+__device__ __forceinline__ void amsgrad_update(float g, float& m, float& v, float& vh, float& th,
+                                               const HyperParams& hp) {
+    m = __fadd_rn(__fmul_rn(hp.beta1, m), __fmul_rn(hp.omb1, g));
+    v = __fadd_rn(__fmul_rn(hp.beta2, v), __fmul_rn(hp.omb2, __fmul_rn(g, g)));
+    vh = fmaxf(vh, v);
+    th = __fsub_rn(th, __fdiv_rn(__fmul_rn(hp.lr, m), __fsqrt_rn(__fadd_rn(vh, hp.eps))));
+}
+
+// gbar = (float)(sum over workers, accumulated in binary64) / (float)n  (Algorithm 2, line 12).
+__device__ __forceinline__ float mean_from_acc(double acc, float nf) {
+    return __fdiv_rn(__double2float_rn(acc), nf);
+}
+
+// Magnitude key: fp32 bits with the sign cleared; unsigned order == order of |x| for finite x.
+__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+// Alignment class of a float pointer: its address in floats modulo 4. Class 0 allows 128-bit
+// accesses, class 2 64-bit ones, odd classes 32-bit ones. Rows of a packed [n, d] buffer start
+// in different classes when d is not a multiple of 4.
+__device__ __forceinline__ int align_class(const void* p) { return (int)((reinterpret_cast<uintptr_t>(p) >> 2) & 3u); }
+
+// Streaming (evict-first) load of 4 consecutive floats at p, whose alignment class is cls.
+__device__ __forceinline__ float4 load4_stream(const float* p, int cls) {
+    float4 r;
+    if (cls == 0) {
+        r = __ldcs(reinterpret_cast<const float4*>(p));
+    } else if (cls == 2) {
+        float2 a = __ldcs(reinterpret_cast<const float2*>(p));
+        float2 b = __ldcs(reinterpret_cast<const float2*>(p + 2));
+        r = make_float4(a.x, a.y, b.x, b.y);
+    } else {
+        r = make_float4(__ldcs(p), __ldcs(p + 1), __ldcs(p + 2), __ldcs(p + 3));
+    }
+    return r;
+}
+
+// Plain (cached) load of 4 consecutive floats.
+__device__ __forceinline__ float4 load4(const float* p, int cls) {
+    float4 r;
+    if (cls == 0) {
+        r = *reinterpret_cast<const float4*>(p);
+    } else if (cls == 2) {
+        float2 a = *reinterpret_cast<const float2*>(p);
+        float2 b = *reinterpret_cast<const float2*>(p + 2);
+        r = make_float4(a.x, a.y, b.x, b.y);
+    } else {
+        r = make_float4(p[0], p[1], p[2], p[3]);
+    }
+    return r;
+}
+
+__device__ __forceinline__ void store4(float* p, int cls, float4 v) {
+    if (cls == 0) {
+        *reinterpret_cast<float4*>(p) = v;
+    } else if (cls == 2) {
+        *reinterpret_cast<float2*>(p) = make_float2(v.x, v.y);
+        *reinterpret_cast<float2*>(p + 2) = make_float2(v.z, v.w);
+    } else {
+        p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
+    }
+}
+
+__device__ __forceinline__ float lane_elem(const float4& v, int k) {
+    return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
+}
+
+// Inclusive scan of one unsigned value per thread across a CTA of kThreads threads.
+// `scratch` holds kWarps words. Returns the inclusive prefix; *total receives the CTA sum.
+__device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t x, uint32_t* scratch, uint32_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t s = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t y = __shfl_up_sync(0xffffffffu, s, o);
+        if (lane >= o) s += y;
+    }
+    __syncthreads();  // scratch may still be read from an earlier call
+    if (lane == 31) scratch[warp] = s;
+    __syncthreads();
+    uint32_t base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        uint32_t c = scratch[w];
+        if (w < warp) base += c;
+        tot += c;
+    }
+    *total = tot;
+    return s + base;
+}
+
+// Deterministic CTA sum of one double per thread (fixed shuffle tree, then warps in order).
+// Result valid in thread 0. `scratch` holds kWarps doubles.
+__device__ __forceinline__ double block_sum_double(double x, double* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = x;
+    __syncthreads();
+    double s = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) s += scratch[w];
+    }
+    return s;
+}
+
+}  // namespace compams

@@ -1,0 +1,203 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2205_05632_b200 import BLOCKSIGN, TOPK, CompAMS, CompAMSError
+from paper_2205_05632_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _pair_run(n, d, offsets, comp, ratio, make_g, steps=4, theta_sigma=0.1, check_e_every=1, **hp):
+    from parity import Pair
+    gen = torch.Generator(device="cuda").manual_seed(1234)
+    p = Pair(n, d, offsets, comp, ratio, **hp)
+    try:
+        p.start(theta_sigma * torch.randn(d, generator=gen, device="cuda"))
+        for t in range(steps):
+            p.step(make_g(gen, t), check_e=(t % check_e_every == 0) or t == steps - 1)
+        return p.inexact
+    finally:
+        p.close()
+
+
+def _randn(n, d):
+    return lambda gen, t: torch.randn(n, d, generator=gen, device="cuda")
+
+
+# ------------------------------------------------------------------ mid-size cases: several tiles, ragged tails
+
+RAGGED = [0, 10, 74, 1098, 5194, 5195, 13387 + 5, 13392 + 3 * 8192 + 1234, 13392 + 3 * 8192 + 1234 + 4097]
+
+
+@pytest.mark.parametrize("n", [1, 3])
+@pytest.mark.parametrize("ratio", [0.01, 0.3, 1.0])
+def test_topk_ragged_blocks(n, ratio):
+    d = RAGGED[-1]
+    _pair_run(n, d, RAGGED, TOPK, ratio, _randn(n, d))
+
+
+@pytest.mark.parametrize("n", [1, 5])
+@pytest.mark.parametrize("check_e_every", [1, 100])
+def test_blocksign_ragged_blocks(n, check_e_every):
+    d = RAGGED[-1]
+    _pair_run(n, d, RAGGED, BLOCKSIGN, 1.0, _randn(n, d), steps=5, check_e_every=check_e_every)
+
+
+@pytest.mark.parametrize("d", [1, 2, 3, 5, 31, 33, 4096, 4097, 8191, 8192, 8193, 3 * 8192 + 2])
+@pytest.mark.parametrize("comp", [TOPK, BLOCKSIGN])
+def test_single_block_sizes_around_tile_edges(d, comp):
+    _pair_run(2, d, [0, d], comp, 0.1, _randn(2, d), steps=3)
+
+
+def test_rows_not_multiple_of_four_use_all_alignment_classes():
+    # d = 1 mod 4: rows 0..3 start at four different 16-byte phases
+    d = 2 * 8192 + 4101
+    for comp in (TOPK, BLOCKSIGN):
+        _pair_run(4, d, [0, 4099, d], comp, 0.05, _randn(4, d), steps=3)
+    _pair_run(4, d, [0, d], TOPK, 1.0, _randn(4, d), steps=3)
+
+
+def test_blocks_of_size_one_and_tiny():
+    d = 200
+    offs = list(range(0, 101)) + [110, 150, 200]
+    for comp in (TOPK, BLOCKSIGN):
+        _pair_run(3, d, offs, comp, 0.2, _randn(3, d), steps=3)
+
+
+# ------------------------------------------------------------------ degenerate inputs: ties everywhere
+
+def _quantised(n, d, levels):
+    def make(gen, t):
+        return torch.randint(-levels, levels + 1, (n, d), generator=gen, device="cuda").float()
+    return make
+
+
+@pytest.mark.parametrize("levels", [0, 1, 3])
+@pytest.mark.parametrize("d,offs", [(3000, [0, 3000]), (40000, [0, 40000]), (60000, [0, 100, 30000, 60000])])
+def test_topk_with_massive_ties(levels, d, offs):
+    # all zeros (levels = 0) or a tiny alphabet: the threshold is tied many times over and the
+    # lower indices must win, tile after tile
+    _pair_run(2, d, offs, TOPK, 0.07, _quantised(2, d, levels), steps=3)
+
+
+def test_topk_ties_straddling_tiles_with_k_one():
+    d = 5 * 8192
+    def make(gen, t):
+        g = torch.zeros(2, d, device="cuda")
+        g[0, 3 * 8192 + 5] = 2.0
+        g[0, 4 * 8192 + 7] = -2.0   # equal magnitude further right: must lose
+        g[1, :] = 1.0
+        return g
+    _pair_run(2, d, [0, d], TOPK, 1.0 / d, make, steps=3)
+
+
+def test_blocksign_zero_and_signed_zero_inputs():
+    d = 10000
+    def make(gen, t):
+        g = torch.randn(2, d, generator=gen, device="cuda")
+        g[0, ::3] = 0.0
+        g[1, ::5] = -0.0
+        if t == 1:
+            g[1] = 0.0
+        return g
+    _pair_run(2, d, [0, 777, d], BLOCKSIGN, 1.0, make, steps=4, check_e_every=2)
+
+
+def test_heavy_tails_and_wide_dynamic_range():
+    d = 50000
+    def make(gen, t):
+        e = torch.randint(-40, 40, (3, d), generator=gen, device="cuda").float()
+        return torch.randn(3, d, generator=gen, device="cuda") * torch.exp2(e)
+    for comp in (TOPK, BLOCKSIGN):
+        _pair_run(3, d, [0, 20000, d], comp, 0.01, make, steps=3)
+
+
+# ------------------------------------------------------------------ reductions
+
+def test_n_one_and_identity_mode_have_zero_error_buffer():
+    d = 3 * 8192 + 77
+    opt = CompAMS(2, d, [0, d], TOPK, 1.0)
+    theta = torch.zeros(d, device="cuda")
+    opt.step(torch.randn(2, d, device="cuda"), theta)
+    assert not opt.buffer("E").any()
+    assert opt.buffer("topk_idx").numel() == 0
+    opt.close()
+
+
+def test_run_to_run_determinism():
+    d = 6 * 8192 + 3
+    G = [torch.randn(4, d, device="cuda") for _ in range(3)]
+    for comp, ratio in ((TOPK, 0.02), (BLOCKSIGN, 1.0)):
+        outs = []
+        for rep in range(2):
+            opt = CompAMS(4, d, [0, 5000, d], comp, ratio)
+            theta = torch.zeros(d, device="cuda")
+            for g in G:
+                opt.step(g, theta)
+            outs.append((theta.clone(), opt.buffer("E").clone(), opt.buffer("vhat").clone()))
+            opt.close()
+        for a, b in zip(*outs):
+            assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+def test_step_host_matches_step():
+    d = 2 * 8192 + 10
+    G = torch.randn(3, d)
+    theta0 = torch.randn(d)
+    a = CompAMS(3, d, [0, d], TOPK, 0.05)
+    b = CompAMS(3, d, [0, d], TOPK, 0.05)
+    th_dev = theta0.cuda()
+    a.step(G.cuda(), th_dev)
+    th_host = theta0.clone()
+    b.step_host(G, th_host)
+    assert torch.equal(th_dev.cpu(), th_host)
+    a.close()
+    b.close()
+
+
+def test_argument_errors_are_reported_not_fatal():
+    with pytest.raises(CompAMSError):
+        CompAMS(0, 10, [0, 10], TOPK, 0.1)
+    with pytest.raises(CompAMSError):
+        CompAMS(2, 10, [0, 5, 5, 10], TOPK, 0.1)
+    with pytest.raises(CompAMSError):
+        CompAMS(2, 10, [0, 10], TOPK, 0.0)
+    with pytest.raises(CompAMSError):
+        CompAMS(2, 10, [0, 10], 7, 0.5)
+    opt = CompAMS(2, 10, [0, 10], TOPK, 0.5)
+    with pytest.raises(CompAMSError):
+        opt.step(torch.zeros(2, 11, device="cuda"), torch.zeros(10, device="cuda"))
+    opt.close()
+
+
+# ------------------------------------------------------------------ the named configurations, 10 chained steps
+
+def test_config1_topk_small_dense_gaussian():
+    from parity import run_workload
+    run_workload(W.config1("cuda"))
+
+
+def test_config2_blocksign_resnet18_shapes():
+    from parity import run_workload
+    run_workload(W.config2("cuda"), check_e_every=3)
+
+
+@pytest.mark.parametrize("ratio", [0.001, 0.01])
+def test_config3_topk_whole_vector_with_zeros(ratio):
+    from parity import run_workload
+    run_workload(W.config3(ratio, "cuda"), check_e_every=3)
+
+
+@pytest.mark.parametrize("comp", [TOPK, BLOCKSIGN])
+def test_config4_resnet50_shapes_layerwise(comp):
+    from parity import run_workload
+    run_workload(W.config4(comp, "cuda"), check_e_every=5)
+
+
+@pytest.mark.parametrize("mode", ["topk", "sign", "dense"])
+@pytest.mark.parametrize("n", [1, 8, 32])
+def test_config5_sweep_points_oracle_sized(mode, n):
+    from parity import run_workload
+    run_workload(W.sweep_point(1 << 20, n, mode, "cuda"), steps=3)
