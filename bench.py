@@ -205,14 +205,10 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the COMP-AMS library has no CPU path")
     from paper_2205_05632_b200 import CompAMS
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2205_05632_b200 import replicas
+    rank, world, local = replicas.rank_world_local()
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dist = replicas.init("nccl", torch.device("cuda", local))
 
     device = "cuda"
     wl = build_workloads(device)
@@ -230,9 +226,7 @@ def main():
             opts[mode].step(wl[mode]["grads"][t % 2], wl[mode]["theta"])
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(dist)
 
     for t in range(args.warmup):
         one_step(t)
@@ -267,14 +261,10 @@ def main():
     for o in opts.values():
         o.check_status()
 
-    if dist is not None:
-        tt = torch.tensor([elapsed_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt[0])
-
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, device)
     ms_per_step = elapsed_ms / args.steps
     elems_per_step = len(MODES) * n * d
-    value = world * elems_per_step / (ms_per_step * 1e-3)
+    value = replicas.aggregate_throughput(elems_per_step, world, ms_per_step)
 
     # ---- roofline of the dominant kernel, live from the event pairs recorded in the timed region
     peak, peak_kind = measured_peak_gbs()
@@ -329,10 +319,7 @@ def main():
                 opts[mode].step_host(host[mode]["g"][t % 2], host[mode]["th"])
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / args.e2e_steps
-        if dist is not None:
-            tt = torch.tensor([dt], device=device, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            dt = float(tt[0])
+        dt = replicas.max_over_ranks(dt, dist, device)
         line["e2e"] = {"value": world * elems_per_step / dt, "unit": UNIT, "ms_per_step": dt * 1e3,
                        "h2d_bytes_per_step": len(MODES) * (n * d * 4 + d * 4),
                        "d2h_bytes_per_step": len(MODES) * d * 4, "steps": args.e2e_steps,
