@@ -47,7 +47,8 @@ enum compams_status {
     COMPAMS_ERR_INVALID_ARG = -1,   /* a null pointer, a size out of range, malformed block offsets ... */
     COMPAMS_ERR_ALLOC = -2,         /* host or device allocation failed */
     COMPAMS_ERR_CUDA = -3,          /* a CUDA runtime call failed (see compams_last_cuda_error) */
-    COMPAMS_ERR_DEVICE_STATUS = -4  /* a kernel recorded an internal inconsistency in the status word */
+    COMPAMS_ERR_DEVICE_STATUS = -4, /* a kernel recorded an internal inconsistency in the status word */
+    COMPAMS_ERR_TOO_LARGE = -5      /* the problem exceeds a fixed capacity (compams_blocksign_sweep_static) */
 };
 
 /* Buffers readable through compams_get_buffer. */
@@ -191,6 +192,48 @@ int compams_get_kernel_time(compams_handle h, int32_t kernel, double* total_ms, 
 
 /* Number of kernel launches the handle has enqueued since creation (all kernels, all steps). */
 int64_t compams_launch_count(compams_handle h);
+
+/*
+ * compams_blocksign_sweep_static - the Block-Sign sweep for callers that cannot allocate device
+ * memory (the paper has no counterpart: this is a packaging of the same arithmetic, not a step
+ * of its algorithms).
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option - inside another framework's
+ * allocator or memory-pool callback, in a process whose device memory was partitioned up front,
+ * or on a latency-critical path where the device-wide synchronisation of an allocation is not
+ * acceptable. compams_create allocates; this call does not: it calls no cudaMalloc, cudaFree or
+ * allocating library routine, and takes every input and output from the caller. Its only scratch
+ * (per-tile partial sums, per-worker arrival counters; 516 KiB) is a fixed array inside the
+ * library's device image, held by every GPU that loads the library until the process exits.
+ *
+ * What it computes, for every worker i over ONE block covering all d coordinates: the corrected
+ * gradient x_i = g_i + e_i (Algorithm 2, line 7), written over x_state; the sign bit of every x_ij;
+ * and the scale ||x_i||_1 / d (Definition 2). The residual of line 8 is deferred exactly as in
+ * compams_step: with deferred != 0, x_state holds the PREVIOUS call's x and scales_prev that call's
+ * scales, and e_i = x_prev - sign(x_prev) * scale_prev is formed on the fly; with deferred == 0,
+ * x_state holds e itself (all zeros before the first step) and scales_prev is not read.
+ *
+ *   grads        device; [n, d] fp32 packed, 4-byte aligned; read only.
+ *   x_state      device; [n, d] fp32 packed, 4-byte aligned; in: e or the previous x; out: x.
+ *   scales_prev  device; [n] fp32; read when deferred != 0 (may be null otherwise). Must not alias scales_out.
+ *   scales_out   device; [n] fp32; receives the scales.
+ *   sign_bits    device; [n, ceil(d/32)] uint32; bit (j % 32) of word j / 32 of row i = sign bit of x_ij;
+ *                unused high bits of a row's last word are 0.
+ *   n, d         1 <= n <= 1024, 1 <= d < 2^31, and n * ceil(d / 8192) <= 65536
+ *                (compams_blocksign_sweep_static_limits returns the two caps); beyond that the call
+ *                does nothing and returns COMPAMS_ERR_TOO_LARGE.
+ *   cuda_stream  a cudaStream_t passed as void* (null = default stream); the work is enqueued there
+ *                and the call returns without synchronising.
+ *
+ * The first call on each device (with that device current) looks up the scratch array's device
+ * address once; make that first call before starting any stream capture. Every call shares the one
+ * array, which keeps the last call's contents (the counters are cleared at the start of each call):
+ * calls whose device work overlaps in time - two streams, two threads - race on it, so serialise them.
+ * Errors: INVALID_ARG (null / misaligned pointer, n or d out of range), TOO_LARGE, CUDA.
+ */
+int compams_blocksign_sweep_static(const float* grads, float* x_state, const float* scales_prev, float* scales_out,
+                                   uint32_t* sign_bits, int32_t n, int64_t d, int32_t deferred, void* cuda_stream);
+int compams_blocksign_sweep_static_limits(int64_t* max_workers, int64_t* max_tiles);
 
 /* Static strings (never null). */
 const char* compams_error_string(int status);

@@ -83,6 +83,10 @@ def load_library() -> ctypes.CDLL:
     L.compams_get_kernel_time.argtypes = [H, c.c_int32, c.POINTER(c.c_double), c.POINTER(c.c_int64)]
     L.compams_launch_count.restype = c.c_int64
     L.compams_launch_count.argtypes = [H]
+    L.compams_blocksign_sweep_static.restype = c.c_int
+    L.compams_blocksign_sweep_static.argtypes = [c.c_void_p] * 5 + [c.c_int32, c.c_int64, c.c_int32, c.c_void_p]
+    L.compams_blocksign_sweep_static_limits.restype = c.c_int
+    L.compams_blocksign_sweep_static_limits.argtypes = [c.POINTER(c.c_int64), c.POINTER(c.c_int64)]
     L.compams_error_string.restype = c.c_char_p
     L.compams_error_string.argtypes = [c.c_int]
     L.compams_kernel_name.restype = c.c_char_p
@@ -99,6 +103,36 @@ def _check(rc: int, what: str) -> None:
         msg = L.compams_error_string(rc).decode()
         cuda = L.compams_last_cuda_error().decode()
         raise CompAMSError("%s failed: %s (%d)%s" % (what, msg, rc, (" [" + cuda + "]") if cuda else ""))
+
+
+def blocksign_sweep_static(grads: torch.Tensor, x_state: torch.Tensor, scales_prev: Optional[torch.Tensor],
+                           scales_out: torch.Tensor, sign_bits: torch.Tensor, deferred: bool,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """compams_blocksign_sweep_static: the Block-Sign sweep over one block per worker row, for callers
+    that cannot allocate device memory. Every buffer is the caller's; nothing is allocated here either
+    (the arguments are passed as raw pointers). See include/compams.h for sizes and limits."""
+    L = load_library()
+    n, d = grads.shape
+    for t in (grads, x_state, scales_out, sign_bits) + ((scales_prev,) if scales_prev is not None else ()):
+        if not (t.is_cuda and t.is_contiguous()):
+            raise CompAMSError("blocksign_sweep_static takes contiguous CUDA tensors")
+    if x_state.shape != grads.shape or scales_out.numel() != n or sign_bits.numel() != n * ((d + 31) // 32):
+        raise CompAMSError("blocksign_sweep_static: buffer shapes do not match [n, d]")
+    s = stream if stream is not None else torch.cuda.current_stream()
+    rc = L.compams_blocksign_sweep_static(
+        ctypes.c_void_p(grads.data_ptr()), ctypes.c_void_p(x_state.data_ptr()),
+        ctypes.c_void_p(scales_prev.data_ptr() if scales_prev is not None else 0),
+        ctypes.c_void_p(scales_out.data_ptr()), ctypes.c_void_p(sign_bits.data_ptr()), int(n), int(d),
+        1 if deferred else 0, ctypes.c_void_p(s.cuda_stream))
+    _check(rc, "compams_blocksign_sweep_static")
+
+
+def blocksign_sweep_static_limits():
+    """(max workers, max n * ceil(d / 8192)) accepted by blocksign_sweep_static."""
+    a, b = ctypes.c_int64(), ctypes.c_int64()
+    _check(load_library().compams_blocksign_sweep_static_limits(ctypes.byref(a), ctypes.byref(b)),
+           "compams_blocksign_sweep_static_limits")
+    return int(a.value), int(b.value)
 
 
 class _DeviceView:

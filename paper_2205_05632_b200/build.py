@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcompams.so")
-SOURCES = ["api.cu", "dense.cu", "blocksign.cu", "topk.cu"]
+SOURCES = ["api.cu", "dense.cu", "blocksign.cu", "topk.cu", "noalloc.cu"]
 HEADERS = ["common.cuh", "context.h", os.path.join("..", "..", "include", "compams.h")]
 
 # -fmad=false: no fused multiply-add anywhere, so each fp32 operation of the update rounds on its own.

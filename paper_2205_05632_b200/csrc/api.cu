@@ -423,6 +423,7 @@ const char* compams_error_string(int status) {
         case COMPAMS_ERR_ALLOC: return "allocation failed";
         case COMPAMS_ERR_CUDA: return "CUDA runtime error";
         case COMPAMS_ERR_DEVICE_STATUS: return "device status word is set";
+        case COMPAMS_ERR_TOO_LARGE: return "problem size exceeds the fixed scratch capacity";
         default: return "unknown status";
     }
 }
