@@ -64,24 +64,28 @@ enum compams_buffer {
     COMPAMS_BUF_SIGN_BITS = 8,    /* uint32 [n, W]   Block-Sign sign bits, see below; W = sum_b ceil(d_b / 32)   */
     COMPAMS_BUF_SIGN_WORD_OFFSETS = 9, /* int64 [M+1] first word of block b inside a row of SIGN_BITS            */
     COMPAMS_BUF_SCALES = 10,      /* float  [n, M]   Block-Sign scales ||x_B||_1 / d_B                           */
-    COMPAMS_BUF_STATUS = 11       /* uint32 [1]      device status word (0 = clean)                              */
+    COMPAMS_BUF_STATUS = 11       /* uint32 [4]      [0] status word (0 = clean); Top-k counters since creation:
+                                                    [1] (worker, block) selections done by the dense passes,
+                                                    [2] selections done inside the candidate list; [3] unused  */
 };
 
 /* Kernel identifiers for compams_get_kernel_time. */
 enum compams_kernel {
     COMPAMS_K_DENSE_MEAN_AMSGRAD = 0, /* k = d: mean over workers fused with the AMSGrad update              */
-    COMPAMS_K_BS_SWEEP = 1,           /* Block-Sign: EF add, block |x| partial sums, sign pack                */
+    COMPAMS_K_BS_SWEEP = 1,           /* Block-Sign: EF add, per-tile |x| sums, sign pack                      */
     COMPAMS_K_BS_APPLY = 2,           /* Block-Sign: segmented average over workers fused with AMSGrad        */
     COMPAMS_K_BS_MATERIALIZE = 3,     /* Block-Sign: turn the stored x into e when E is read                  */
-    COMPAMS_K_TOPK_SWEEP = 4,         /* Top-k: EF add, x written to E, first radix histogram                 */
-    COMPAMS_K_TOPK_HIST = 5,          /* Top-k: later radix histogram passes                                  */
-    COMPAMS_K_TOPK_FIND = 6,          /* Top-k: locate the threshold bin of a pass                            */
-    COMPAMS_K_TOPK_COLLECT = 7,       /* Top-k: emit (index, value), zero kept e, count threshold ties        */
-    COMPAMS_K_TOPK_TIES = 8,          /* Top-k: take the lowest-index ties at the threshold                   */
+    COMPAMS_K_TOPK_SWEEP = 4,         /* Top-k: EF add, x written to E, candidates above the predicted threshold */
+    COMPAMS_K_TOPK_HIST = 5,          /* Top-k dense passes: radix histograms over x                          */
+    COMPAMS_K_TOPK_FIND = 6,          /* Top-k dense passes: locate the threshold bin of a pass               */
+    COMPAMS_K_TOPK_COLLECT = 7,       /* Top-k dense passes: emit (index, value), count threshold ties        */
+    COMPAMS_K_TOPK_TIES = 8,          /* Top-k: lowest-index ties at the threshold; closes the step per segment */
     COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: sparse scatter-accumulate into the averaged gradient          */
     COMPAMS_K_AMSGRAD = 10,           /* Top-k: AMSGrad update from the accumulated average                   */
     COMPAMS_K_TOPK_SMALL = 11,        /* Top-k: whole small blocks selected inside shared memory              */
-    COMPAMS_K_COUNT = 12
+    COMPAMS_K_TOPK_SELECT = 12,       /* Top-k: exact selection inside the candidate lists                    */
+    COMPAMS_K_BS_SCALES = 13,         /* Block-Sign: scale of every (worker, block) from the tile sums        */
+    COMPAMS_K_COUNT = 14
 };
 
 /*

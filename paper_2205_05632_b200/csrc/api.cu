@@ -63,32 +63,69 @@ int64_t kept_per_block(double k_ratio, int64_t d_b) {
     return k;
 }
 
-// Cuts the listed blocks into tiles of kTile coordinates and uploads the tables.
-int build_tiles(compams_context* c, const std::vector<int32_t>& blocks) {
-    std::vector<int32_t> tile_blk, tile_r0, tile_seg, seg_tile0;
-    seg_tile0.push_back(0);
+// Cuts the listed blocks into tiles of kTile coordinates and uploads the tile and segment tables.
+// For Top-k (`topk` true) every listed block also gets its message slots and candidate capacity.
+int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool topk) {
+    std::vector<TileInfo> tiles;
+    std::vector<SegInfo> segs;
+    int64_t cand_total = 0;
     for (size_t s = 0; s < blocks.size(); ++s) {
         const int32_t b = blocks[s];
         const int64_t len = c->off[b + 1] - c->off[b];
-        for (int64_t r0 = 0; r0 < len; r0 += kTile) {
-            tile_blk.push_back(b);
-            tile_r0.push_back((int32_t)r0);
-            tile_seg.push_back((int32_t)s);
+        const int64_t nt = (len + kTile - 1) / kTile;
+        if ((int64_t)tiles.size() + nt > (int64_t)0x7fffffff) return COMPAMS_ERR_INVALID_ARG;
+        SegInfo si{};
+        si.o = c->off[b];
+        si.len = (int32_t)len;
+        si.blk = b;
+        si.tile0 = (int32_t)tiles.size();
+        si.ntile_b = (int32_t)nt;
+        if (topk) {
+            const int64_t kb = c->seg_off[(size_t)b + 1] - c->seg_off[(size_t)b];
+            si.slot0 = c->seg_off[(size_t)b];
+            si.kb = (uint32_t)kb;
+            // the candidate path pays off for sparse selections only: at most 1/32 of the block kept
+            int64_t cap = (kb * 32 <= len) ? 8 * kb + 1024 : 0;
+            if (cap > len) cap = len;
+            si.cap = (uint32_t)cap;
+            si.cand_off = cand_total;
+            cand_total += cap;
         }
-        if (tile_blk.size() > (size_t)0x7fffffff) return COMPAMS_ERR_INVALID_ARG;
-        seg_tile0.push_back((int32_t)tile_blk.size());
+        for (int64_t r0 = 0; r0 < len; r0 += kTile) {
+            TileInfo ti{};
+            ti.o = c->off[b];
+            ti.len = (int32_t)len;
+            ti.r0 = (int32_t)r0;
+            ti.blk = b;
+            ti.seg = (int32_t)s;
+            ti.tile0 = si.tile0;
+            ti.ntile_b = si.ntile_b;
+            tiles.push_back(ti);
+        }
+        segs.push_back(si);
     }
-    int32_t *d_blk, *d_r0, *d_seg, *d_t0;
-    RC(dev_upload(c, &d_blk, tile_blk));
-    RC(dev_upload(c, &d_r0, tile_r0));
-    RC(dev_upload(c, &d_seg, tile_seg));
-    RC(dev_upload(c, &d_t0, seg_tile0));
-    c->tab.ntiles = (int32_t)tile_blk.size();
-    c->tab.tile_blk = d_blk;
-    c->tab.tile_r0 = d_r0;
-    c->tab.tile_seg = d_seg;
-    c->tab.seg_tile0 = d_t0;
+    TileInfo* d_tiles;
+    SegInfo* d_segs;
+    RC(dev_upload(c, &d_tiles, tiles));
+    RC(dev_upload(c, &d_segs, segs));
+    c->tab.ntiles = (int32_t)tiles.size();
+    c->tab.tiles = d_tiles;
     c->tab.nseg = (int32_t)blocks.size();
+    c->tab.segs = d_segs;
+    c->tk.cand_total = cand_total;
+    c->seg_cap_host.clear();
+    for (const SegInfo& si : segs) c->seg_cap_host.push_back(si.cap);
+    if (topk) {
+        std::vector<int32_t> small_l, big_l;
+        for (size_t s = 0; s < segs.size(); ++s) {
+            if (segs[s].cap == 0) continue;  // never predicts: always the dense passes, no select needed
+            (segs[s].cap <= (uint32_t)kSelectSingleMax ? small_l : big_l).push_back((int32_t)s);
+        }
+        RC(dev_upload(c, &c->sel_small, small_l));
+        RC(dev_upload(c, &c->sel_big, big_l));
+        c->n_sel_small = (int)small_l.size();
+        c->n_sel_big = (int)big_l.size();
+    }
     return COMPAMS_OK;
 }
 
@@ -108,7 +145,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
     RC(dev_alloc(c, &c->v, (size_t)d));
     RC(dev_alloc(c, &c->vhat, (size_t)d));
     RC(dev_alloc(c, &c->gbar, (size_t)d));
-    RC(dev_alloc(c, &c->status, 1));
+    RC(dev_alloc(c, &c->status, 4));
 
     if (c->compressor == COMPAMS_TOPK) {
         c->seg_off.assign((size_t)M + 1, 0);
@@ -131,7 +168,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_upload(c, &c->d_seg_off, c->seg_off));
         std::vector<int32_t> small, large;
         for (int32_t b = 0; b < M; ++b) ((c->off[b + 1] - c->off[b] <= kSmallMax) ? small : large).push_back(b);
-        RC(build_tiles(c, large));
+        RC(build_tiles(c, large, true));
         TopkBuffers& t = c->tk;
         t.E = c->E;
         t.K = c->K;
@@ -143,8 +180,21 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &t.idx, (size_t)n * (size_t)c->K));
         RC(dev_alloc(c, &t.val, (size_t)n * (size_t)c->K));
         RC(dev_alloc(c, &t.hist, (size_t)n * (size_t)c->tab.nseg * kBins1));
-        RC(dev_alloc(c, &t.seg, (size_t)n * (size_t)c->tab.nseg));
+        {
+            SegState init{};
+            init.tau_hat = kNoPrediction;
+            init.tau_prev = kNoPrediction;
+            std::vector<SegState> seg0((size_t)n * (size_t)c->tab.nseg, init);
+            uint32_t never = 0;
+            for (uint32_t cap : c->seg_cap_host) never += cap ? 0u : 1u;
+            for (size_t k = 0; k < seg0.size(); ++k)
+                seg0[k].fallback = c->seg_cap_host[k % (size_t)c->tab.nseg] ? 0u : 1u;
+            RC(dev_upload(c, &t.seg, seg0));
+            std::vector<uint32_t> dc(1, never * (uint32_t)n);
+            RC(dev_upload(c, &t.dense_count, dc));
+        }
         RC(dev_alloc(c, &t.tile_ties, (size_t)n * (size_t)c->tab.ntiles));
+        RC(dev_alloc(c, &t.cand, (size_t)n * (size_t)t.cand_total, false));
         RC(dev_alloc(c, &t.acc, (size_t)d));
         t.status = c->status;
         t.gbar = c->gbar;
@@ -155,7 +205,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &c->E, (size_t)n * (size_t)d));
         std::vector<int32_t> all((size_t)M);
         for (int32_t b = 0; b < M; ++b) all[(size_t)b] = b;
-        RC(build_tiles(c, all));
+        RC(build_tiles(c, all, false));
         std::vector<int64_t> word_off((size_t)M + 1, 0);
         for (int32_t b = 0; b < M; ++b)
             word_off[(size_t)b + 1] = word_off[(size_t)b] + (c->off[b + 1] - c->off[b] + 31) / 32;
@@ -169,7 +219,6 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &c->scales[0], (size_t)n * (size_t)M));
         RC(dev_alloc(c, &c->scales[1], (size_t)n * (size_t)M));
         RC(dev_alloc(c, &s.tile_sum, (size_t)n * (size_t)c->tab.ntiles));
-        RC(dev_alloc(c, &s.ticket, (size_t)n * (size_t)M));
         s.gbar = c->gbar;
         s.m = c->m;
         s.v = c->v;
@@ -222,12 +271,15 @@ int step_device(compams_context* c, const float* grads, float* theta) {
         c->scales_cur ^= 1;
         RC(run_kernel(c, COMPAMS_K_BS_SWEEP, [&] { return launch_bs_sweep(c, grads); }));
         c->e_is_x = true;
+        RC(run_kernel(c, COMPAMS_K_BS_SCALES, [&] { return launch_bs_scales(c); }));
         RC(run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); }));
         return COMPAMS_OK;
     }
     if (c->tk.nsmall > 0) RC(run_kernel(c, COMPAMS_K_TOPK_SMALL, [&] { return launch_topk_small(c, grads); }));
     if (c->tab.ntiles > 0) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_SELECT, [&] { return launch_topk_select(c); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 1); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 1); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 2); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 2); }));
@@ -372,7 +424,7 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
         case COMPAMS_BUF_SIGN_BITS: if (sign) { p = c->bs.bits; cnt = (int64_t)c->n * c->W; } break;
         case COMPAMS_BUF_SIGN_WORD_OFFSETS: if (sign) { p = c->d_word_off; cnt = c->M + 1; } break;
         case COMPAMS_BUF_SCALES: if (sign) { p = c->scales[c->scales_cur]; cnt = (int64_t)c->n * c->M; } break;
-        case COMPAMS_BUF_STATUS: p = c->status; cnt = 1; break;
+        case COMPAMS_BUF_STATUS: p = c->status; cnt = 4; break;
         default: return COMPAMS_ERR_INVALID_ARG;
     }
     *dev_ptr = p;
@@ -431,7 +483,7 @@ const char* compams_error_string(int status) {
 const char* compams_kernel_name(int32_t kernel) {
     static const char* names[COMPAMS_K_COUNT] = {
         "dense_mean_amsgrad", "bs_sweep", "bs_apply", "bs_materialize", "topk_sweep", "topk_hist",
-        "topk_find", "topk_collect", "topk_ties", "topk_scatter", "amsgrad", "topk_small"};
+        "topk_find", "topk_collect", "topk_ties", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
     return (kernel >= 0 && kernel < COMPAMS_K_COUNT) ? names[kernel] : "unknown";
 }
 

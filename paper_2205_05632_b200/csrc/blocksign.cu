@@ -1,8 +1,9 @@
 // Block-Sign path (Definition 2) of the COMP-AMS step.
 //
 // bs_sweep   per (worker, tile): x = g + e (Algorithm 2, line 7), x written over E, sign bits
-//            packed, sum |x| of the tile in binary64. The last tile of a (worker, block) to
-//            finish adds the tile sums in a fixed order and writes the scale ||x_B||_1 / d_B.
+//            packed, sum |x| of the tile in binary64.
+// bs_scales  per (worker, block): adds the tile sums in a fixed order and writes the scale
+//            ||x_B||_1 / d_B.
 // bs_apply   per coordinate: gbar = (1/n) sum_i sign(x_ij) s_{i,b} from the sign bits and
 //            scales (line 12), fused with the AMSGrad update (lines 13-16).
 //
@@ -24,17 +25,24 @@ __device__ __forceinline__ uint32_t pack_group_word(uint32_t nibble, int lane) {
     return w;
 }
 
+// |x| as a binary64 number without a conversion instruction: for a normal fp32 value the
+// binary64 pattern is the same fraction shifted left by 29 bits under an exponent rebiased by 896.
+__device__ __forceinline__ double abs_as_double(float x) {
+    const uint32_t b = __float_as_uint(x) & 0x7fffffffu;
+    if ((b >> 23) == 0u) return (double)__uint_as_float(b);  // zero or subnormal: rare, take the conversion
+    return __hiloint2double((int)((b >> 3) + 0x38000000u), (int)(b << 29));
+}
+
 template <bool FULL>
-__device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int64_t len,
-                                              int64_t rw, int lane, bool deferred, float sp, double& acc,
-                                              uint32_t& myword) {
+__device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int rw,
+                                              int lane, bool deferred, float sp, double& acc, uint32_t& myword) {
     const int cg = align_class(g), ce = align_class(e);
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        float4 gv[4], ev[4];
+    for (int bt = 0; bt < kIters / 2; ++bt) {
+        float4 gv[2], ev[2];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t r = rw + (half * 4 + u) * 128 + lane * 4;
+        for (int u = 0; u < 2; ++u) {
+            const int r = rw + (bt * 2 + u) * 128 + lane * 4;
             if (FULL || r + 3 < len) {
                 gv[u] = load4_stream(g + r, cg);
                 ev[u] = load4_stream(e + r, ce);
@@ -50,9 +58,9 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int it = half * 4 + u;
-            const int64_t r = rw + it * 128 + lane * 4;
+        for (int u = 0; u < 2; ++u) {
+            const int it = bt * 2 + u;
+            const int r = rw + it * 128 + lane * 4;
             float xs[4];
             uint32_t nib = 0;
 #pragma unroll
@@ -64,7 +72,7 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
                 xs[k] = x;
                 const bool live = FULL || (r + k < len);
                 if (live) {
-                    acc += (double)fabsf(x);
+                    acc += abs_as_double(x);
                     nib |= (__float_as_uint(x) >> 31) << k;
                 }
             }
@@ -82,65 +90,56 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
     }
 }
 
-__global__ void __launch_bounds__(kThreads) bs_sweep_kernel(Tables t, BsBuffers b, const float* __restrict__ G,
-                                                            int deferred) {
+__global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffers b, const float* __restrict__ G,
+                                                               int deferred) {
     __shared__ double red[kWarps];
-    __shared__ int is_last;
     const int tile = blockIdx.x;
     const int i = blockIdx.y;
-    const int blk = t.tile_blk[tile];
-    const int64_t o = t.off[blk];
-    const int64_t len = t.off[blk + 1] - o;
-    const int64_t r0 = t.tile_r0[tile];
+    const TileInfo ti = load_tile(t.tiles, tile);
+    const int blk = ti.blk;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float* g = G + (size_t)i * (size_t)t.d + (size_t)o;
-    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
+    const float* g = G + (size_t)i * (size_t)t.d + (size_t)ti.o;
+    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
     const float sp = deferred ? b.scales_prev[(size_t)i * t.M + blk] : 0.0f;
-    const int64_t rw = r0 + (int64_t)warp * kWarpSpan;
+    const int rw = ti.r0 + warp * kWarpSpan;
 
     double acc = 0.0;
     uint32_t myword = 0;
-    if (r0 + kTile <= len)
-        bs_sweep_tile<true>(g, e, len, rw, lane, deferred != 0, sp, acc, myword);
+    if (ti.r0 + kTile <= ti.len)
+        bs_sweep_tile<true>(g, e, ti.len, rw, lane, deferred != 0, sp, acc, myword);
     else
-        bs_sweep_tile<false>(g, e, len, rw, lane, deferred != 0, sp, acc, myword);
+        bs_sweep_tile<false>(g, e, ti.len, rw, lane, deferred != 0, sp, acc, myword);
 
-    if (rw + (int64_t)lane * 32 < len)
+    if (rw + lane * 32 < ti.len)
         b.bits[(size_t)i * (size_t)b.W + (size_t)b.word_off[blk] + (size_t)(rw >> 5) + lane] = myword;
 
-    // tile sum, then "last tile to arrive finalises the block" (no waiting on other CTAs)
+    // tile sum in binary64 (fixed shuffle tree); bs_scales adds the tile sums of a block in a fixed order
     double s = block_sum_double(acc, red);
-    const int tile0 = t.seg_tile0[blk];
-    const int ntile_b = t.seg_tile0[blk + 1] - tile0;
-    if (threadIdx.x == 0) {
-        b.tile_sum[(size_t)i * t.ntiles + tile] = s;
-        __threadfence();
-        uint32_t ticket = atomicAdd(&b.ticket[(size_t)i * t.M + blk], 1u);
-        is_last = (ticket == (uint32_t)(ntile_b - 1));
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
+    if (threadIdx.x == 0) b.tile_sum[(size_t)i * t.ntiles + tile] = s;
+}
+
+// One CTA per (worker, block): scale = ||x_B||_1 / d_B from the tile sums (Definition 2).
+__global__ void __launch_bounds__(kThreads) bs_scales_kernel(Tables t, BsBuffers b) {
+    __shared__ double red[kWarps];
+    const int blk = blockIdx.x, i = blockIdx.y;
+    const SegInfo* si = t.segs + blk;
+    const double* ts = b.tile_sum + (size_t)i * t.ntiles + si->tile0;
     double part = 0.0;
-    const double* ts = b.tile_sum + (size_t)i * t.ntiles + tile0;
-    for (int k = threadIdx.x; k < ntile_b; k += kThreads) part += __ldcg(ts + k);
-    double S = block_sum_double(part, red);
-    if (threadIdx.x == 0) {
-        // Definition 2: scale = ||x_B||_1 / d_B, one division in binary64, one rounding to fp32
-        b.scales_cur[(size_t)i * t.M + blk] = __double2float_rn(S / (double)len);
-        b.ticket[(size_t)i * t.M + blk] = 0u;
-    }
+    for (int k = threadIdx.x; k < si->ntile_b; k += kThreads) part += ts[k];
+    const double S = block_sum_double(part, red);
+    // one division in binary64, one rounding to fp32
+    if (threadIdx.x == 0) b.scales_cur[(size_t)i * t.M + blk] = __double2float_rn(S / (double)si->len);
 }
 
 // E holds x; turn it into e = x - sign(x) * s in place (Algorithm 2, line 8).
 __global__ void __launch_bounds__(kThreads) bs_materialize_kernel(Tables t, float* __restrict__ E,
                                                                   const float* __restrict__ scales) {
-    const int tile = blockIdx.x;
     const int i = blockIdx.y;
-    const int blk = t.tile_blk[tile];
-    const int64_t o = t.off[blk];
-    const int64_t len = t.off[blk + 1] - o;
-    const int64_t r0 = t.tile_r0[tile];
+    const TileInfo ti = load_tile(t.tiles, blockIdx.x);
+    const int blk = ti.blk;
+    const int64_t o = ti.o;
+    const int64_t len = ti.len;
+    const int64_t r0 = ti.r0;
     const float s = scales[(size_t)i * t.M + blk];
     float* e = E + (size_t)i * (size_t)t.d + (size_t)o;
     const int64_t end = (r0 + kTile < len) ? r0 + kTile : len;
@@ -156,11 +155,11 @@ __global__ void __launch_bounds__(kThreads) bs_apply_kernel(Tables t, BsBuffers 
                                                             HyperParams hp) {
     __shared__ uint32_t sh_bits[kApplyChunk][kTile / 32];
     __shared__ double sh_s[kApplyChunk];
-    const int tile = blockIdx.x;
-    const int blk = t.tile_blk[tile];
-    const int64_t o = t.off[blk];
-    const int64_t len = t.off[blk + 1] - o;
-    const int64_t r0 = t.tile_r0[tile];
+    const TileInfo ti = load_tile(t.tiles, blockIdx.x);
+    const int blk = ti.blk;
+    const int64_t o = ti.o;
+    const int64_t len = ti.len;
+    const int64_t r0 = ti.r0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t rw = r0 + (int64_t)warp * kWarpSpan;
 
@@ -240,6 +239,14 @@ cudaError_t launch_bs_sweep(compams_context* c, const float* grads) {
     b.scales_prev = c->scales[c->scales_cur ^ 1];
     b.scales_cur = c->scales[c->scales_cur];
     bs_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, grads, c->e_is_x ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bs_scales(compams_context* c) {
+    dim3 grid((unsigned)c->M, (unsigned)c->n);
+    BsBuffers b = c->bs;
+    b.scales_cur = c->scales[c->scales_cur];
+    bs_scales_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b);
     return cudaGetLastError();
 }
 

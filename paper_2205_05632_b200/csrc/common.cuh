@@ -12,6 +12,30 @@ constexpr int kTile = 8192;            // coordinates per tile: 8 warps x 8 iter
 constexpr int kWarpSpan = kTile / kWarps;  // 1024 consecutive coordinates per warp
 constexpr int kIters = kWarpSpan / 128;    // 8 iterations of one float4 per lane
 
+// One tile: kTile consecutive coordinates of one block (the last tile of a block may be shorter).
+struct __align__(16) TileInfo {
+    int64_t o;        // first coordinate of the block inside [0, d)
+    int32_t len;      // block length d_b
+    int32_t r0;       // first coordinate of the tile, relative to the block
+    int32_t blk;      // block index b
+    int32_t seg;      // index of the block among the tiled blocks
+    int32_t tile0;    // first tile of the block
+    int32_t ntile_b;  // number of tiles of the block
+};
+
+// One tiled block as the kernels see it (the Top-k fields are 0 for Block-Sign).
+struct __align__(16) SegInfo {
+    int64_t o;         // first coordinate of the block
+    int64_t slot0;     // first message slot of the block inside a worker's row of K entries
+    int64_t cand_off;  // first candidate slot of the block inside a worker's row of candidate slots
+    int32_t len;       // block length d_b
+    int32_t blk;       // block index b
+    int32_t tile0;     // first tile
+    int32_t ntile_b;   // number of tiles
+    uint32_t kb;       // entries to keep
+    uint32_t cap;      // candidate capacity (0: this block never uses the candidate path)
+};
+
 // AMSGrad hyper-parameters as the fp32 numbers every kernel uses (Algorithm 1).
 struct HyperParams {
     float lr, beta1, beta2, omb1, omb2, eps, nf;  // omb = 1 - beta (fp32), nf = (float)n
@@ -83,6 +107,21 @@ __device__ __forceinline__ void store4(float* p, int cls, float4 v) {
 
 __device__ __forceinline__ float lane_elem(const float4& v, int k) {
     return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
+}
+
+// Tile record `tile` of a table, fetched with two 128-bit read-only loads.
+__device__ __forceinline__ TileInfo load_tile(const TileInfo* tiles, int tile) {
+    const int4* p = reinterpret_cast<const int4*>(tiles + tile);
+    const int4 a = __ldg(p), b = __ldg(p + 1);
+    TileInfo ti;
+    ti.o = ((int64_t)(uint32_t)a.y << 32) | (uint32_t)a.x;
+    ti.len = a.z;
+    ti.r0 = a.w;
+    ti.blk = b.x;
+    ti.seg = b.y;
+    ti.tile0 = b.z;
+    ti.ntile_b = b.w;
+    return ti;
 }
 
 // Inclusive scan of one unsigned value per thread across a CTA of kThreads threads.

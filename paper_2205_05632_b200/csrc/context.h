@@ -16,8 +16,22 @@ constexpr int kBins1 = 2048;       // radix pass 1: key bits 30..20
 constexpr int kBins23 = 1024;      // radix passes 2, 3: key bits 19..10, 9..0
 constexpr int kMaxTimed = 4096;    // event pairs kept for per-kernel timing
 
-// Per (worker, large block) Top-k selection state, written by the find kernels.
+constexpr uint32_t kNoPrediction = 0xffffffffu;  // tau_hat value that no key reaches
+constexpr int kTileCand = 1024;          // candidates one tile can stage in shared memory
+constexpr int kSelectCluster = 8;        // CTAs cooperating on one long candidate list
+constexpr int kSelBins = 4096;           // bins of the candidate select's first histogram
+constexpr int kSelectSingleMax = 24576;  // candidate capacity up to which one CTA handles a segment
+
+// Per (worker, large block) Top-k selection state.
 struct SegState {
+    // candidate path
+    uint32_t tau_hat;     // keys >= tau_hat are collected as candidates by the sweep (kNoPrediction: none)
+    uint32_t tau_prev;    // threshold key of the previous step (kNoPrediction: unknown)
+    uint32_t cand_count;  // candidates counted by the sweep (may exceed what was stored)
+    uint32_t sel_shift;   // log2 of the bin width of the select's first histogram
+    uint32_t fallback;    // 1: the candidate path could not decide this step, the dense passes run
+    uint32_t edge;        // dense path: bin edge chosen as the next tau_hat
+    // dense radix passes
     uint32_t prefix;      // high key bits decided so far
     uint32_t k_rem;       // entries still to take among the keys that match the prefix
     uint32_t tau;         // threshold key (after the last pass)
@@ -25,7 +39,7 @@ struct SegState {
     uint32_t ties_take;   // how many of them belong to the kept set
     uint32_t need_order;  // 1 when ties_take < ties_total: the lowest indices must be chosen
     uint32_t emit_count;  // message slots handed out so far
-    uint32_t pad;
+    uint32_t pad[3];
 };
 
 // Block / tile tables shared by the tiled kernels (device pointers).
@@ -33,14 +47,11 @@ struct Tables {
     int32_t n;
     int64_t d;
     int32_t M;
-    const int64_t* off;        // [M+1] block offsets
-    // tiles: every listed block is cut into tiles of kTile coordinates
-    int32_t ntiles;            // tiles per worker row
-    const int32_t* tile_blk;   // [ntiles] block index b of the tile
-    const int32_t* tile_r0;    // [ntiles] first coordinate of the tile, relative to its block
-    const int32_t* tile_seg;   // [ntiles] index of the block among the tiled blocks
-    const int32_t* seg_tile0;  // [nseg+1] first tile of each tiled block
-    int32_t nseg;              // number of tiled blocks (all blocks for Block-Sign, large ones for Top-k)
+    const int64_t* off;     // [M+1] block offsets
+    int32_t ntiles;         // tiles per worker row
+    const TileInfo* tiles;  // [ntiles]
+    int32_t nseg;           // number of tiled blocks (all blocks for Block-Sign, large ones for Top-k)
+    const SegInfo* segs;    // [nseg]
 };
 
 struct BsBuffers {
@@ -51,7 +62,6 @@ struct BsBuffers {
     const float* scales_prev; // [n, M]
     float* scales_cur;        // [n, M]
     double* tile_sum;         // [n, ntiles]
-    uint32_t* ticket;         // [n, M]
     float *gbar, *m, *v, *vhat;
 };
 
@@ -66,6 +76,9 @@ struct TopkBuffers {
     uint32_t* hist;            // [n * nseg, kBins1]
     SegState* seg;             // [n * nseg]
     uint32_t* tile_ties;       // [n, ntiles]
+    uint2* cand;               // [n, cand_total] (coordinate, bits of x) pairs collected by the sweep
+    int64_t cand_total;        // candidate slots per worker
+    uint32_t* dense_count;     // [1] segments currently marked for the dense passes
     double* acc;               // [d] binary64 accumulator of the worker average
     uint32_t* status;
     float *gbar, *m, *v, *vhat;
@@ -87,12 +100,16 @@ struct compams_context {
 
     std::vector<int64_t> off;      // host copy of the block offsets
     std::vector<int64_t> seg_off;  // host prefix sums of k_b (Top-k)
+    std::vector<uint32_t> seg_cap_host;  // candidate capacity of every tiled block (Top-k)
     int64_t K = 0;
     int64_t W = 0;
 
     compams::Tables tab{};
     compams::BsBuffers bs{};
     compams::TopkBuffers tk{};
+    int32_t* sel_small = nullptr;  // tiled blocks whose candidate lists one CTA selects from
+    int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists a cluster selects from
+    int n_sel_small = 0, n_sel_big = 0;
     float* scales[2] = {nullptr, nullptr};
     int scales_cur = 0;
     bool e_is_x = false;  // Block-Sign: E holds the corrected gradient x of the last step, not e
@@ -122,10 +139,12 @@ namespace compams {
 // Each launcher enqueues one kernel on ctx->stream and returns the launch status.
 cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, float* theta);
 cudaError_t launch_bs_sweep(compams_context* c, const float* grads);
+cudaError_t launch_bs_scales(compams_context* c);
 cudaError_t launch_bs_apply(compams_context* c, float* theta);
 cudaError_t launch_bs_materialize(compams_context* c);
 cudaError_t launch_topk_small(compams_context* c, const float* grads);
 cudaError_t launch_topk_sweep(compams_context* c, const float* grads);
+cudaError_t launch_topk_select(compams_context* c);
 cudaError_t launch_topk_hist(compams_context* c, int pass);
 cudaError_t launch_topk_find(compams_context* c, int pass);
 cudaError_t launch_topk_collect(compams_context* c);

@@ -7,50 +7,45 @@
 //   Blocks of at most kSmallMax coordinates: topk_small - one CTA holds the block in shared
 //   memory and does every radix pass there; E is written once.
 //
-//   Larger blocks, cut into tiles of kTile coordinates:
-//     topk_sweep    x = g + e written over E (Algorithm 2, line 7), histogram of key bits 30..20
-//     topk_find     threshold bin of the pass just histogrammed; narrows (prefix, k_rem)
-//     topk_hist     histogram of the next 10 key bits among the keys that match the prefix
-//     topk_collect  after the last find: keys above the threshold are emitted as (index, value);
-//                   threshold ties are emitted too unless only some of them fit, in which case
-//                   they are counted per tile
-//     topk_ties     takes the lowest-index threshold ties, tile by tile in index order
+//   Larger blocks, cut into tiles of kTile coordinates.
+//   Candidate path (one pass over [n, d]):
+//     topk_sweep    x = g + e written over E (Algorithm 2, line 7); every key >= tau_hat, a threshold
+//                   predicted from the previous step, is appended to the segment's candidate list
+//     topk_select   one CTA (short lists) or a cluster of 8 CTAs (long lists) per segment: if the list
+//                   holds at least k_b and at most its capacity, the exact Top-k is inside it. A
+//                   histogram of the key offsets above tau_hat (bins sized from the last step, merged
+//                   through distributed shared memory) finds the threshold bin; winners above it are
+//                   emitted, the bin's few candidates go to shared memory and a radix select over
+//                   (low key bits, ~index) composites finishes the job and predicts the next tau_hat.
+//                   Otherwise the segment is marked for the dense passes.
+//   Dense passes (only for marked segments; exact for any input, e.g. all-equal values):
+//     topk_hist<1..3> / topk_find<1..3>  three histogram passes over x, 11 + 10 + 10 key bits
+//     topk_collect  keys above the threshold are emitted; threshold ties too unless only some fit,
+//                   in which case they are counted per tile
+//     topk_ties     takes the lowest-index threshold ties, tile by tile in index order; also closes
+//                   the step for every segment (count check, counters reset)
 //   topk_scatter    walks the (index, value) messages: sum_i g~_i accumulated into a binary64
 //                   buffer (line 12) and e zeroed at every kept coordinate (line 8: e = x - x)
+#include <cooperative_groups.h>
+
 #include "context.h"
+
+namespace cg = cooperative_groups;
 
 namespace compams {
 
 // ------------------------------------------------------------------------------------------
-// tile loads shared by the large-block kernels
+// tile addressing shared by the large-block kernels
 
-struct TileCoord {
-    int i, tile, seg, blk;
-    int64_t o, len, r0;
-    size_t sg;  // i * nseg + seg
-};
-
-__device__ __forceinline__ TileCoord tile_coord(const Tables& t, int i, int tile) {
-    TileCoord c;
-    c.i = i;
-    c.tile = tile;
-    c.seg = t.tile_seg[tile];
-    c.blk = t.tile_blk[tile];
-    c.o = t.off[c.blk];
-    c.len = t.off[c.blk + 1] - c.o;
-    c.r0 = t.tile_r0[tile];
-    c.sg = (size_t)i * t.nseg + c.seg;
-    return c;
-}
-
-// Coordinates of lane `lane` of warp `warp` at iteration `it`: 4 consecutive ones starting here.
-__device__ __forceinline__ int64_t lane_r(int64_t r0, int warp, int it, int lane) {
-    return r0 + (int64_t)warp * kWarpSpan + it * 128 + lane * 4;
+// First of the 4 consecutive coordinates (relative to the block) that lane `lane` of warp `warp`
+// handles at iteration `it` of a tile starting at r0.
+__device__ __forceinline__ int lane_r(int r0, int warp, int it, int lane) {
+    return r0 + warp * kWarpSpan + it * 128 + lane * 4;
 }
 
 // Loads the 32 values of this thread's share of a tile of x (already stored in E).
-// Coordinates past the block end read as +0 (callers mask them with `live`).
-__device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int64_t len, int64_t r0, int warp, int lane,
+// Coordinates past the block end read as +0 (callers mask them).
+__device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int len, int r0, int warp, int lane,
                                             float4 (&xv)[kIters]) {
     const int ce = align_class(e);
     if (r0 + kTile <= len) {
@@ -59,7 +54,7 @@ __device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int64_t
     } else {
 #pragma unroll
         for (int it = 0; it < kIters; ++it) {
-            const int64_t r = lane_r(r0, warp, it, lane);
+            const int r = lane_r(r0, warp, it, lane);
             if (r + 3 < len) {
                 xv[it] = load4(e + r, ce);
             } else {
@@ -73,20 +68,22 @@ __device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int64_t
 }
 
 // ------------------------------------------------------------------------------------------
-// sweep: x = g + e -> E, histogram of the top 11 key bits
+// sweep: x = g + e -> E; keys >= tau_hat go to the candidate list
 
 template <bool FULL>
-__device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int64_t len,
-                                                int64_t r0, int warp, int lane, uint32_t* sh) {
-    const int cg = align_class(g), ce = align_class(e);
+__device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int r0,
+                                                int warp, int lane, uint32_t tau_hat, uint32_t coord0,
+                                                uint2* sh_cand, uint32_t* sh_cnt, uint32_t* g_cnt, uint2* g_out,
+                                                uint32_t cap) {
+    const int cg_ = align_class(g), ce = align_class(e);
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        float4 gv[4], ev[4];
+    for (int bt = 0; bt < kIters / 2; ++bt) {
+        float4 gv[2], ev[2];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t r = lane_r(r0, warp, half * 4 + u, lane);
+        for (int u = 0; u < 2; ++u) {
+            const int r = lane_r(r0, warp, bt * 2 + u, lane);
             if (FULL || r + 3 < len) {
-                gv[u] = load4_stream(g + r, cg);
+                gv[u] = load4_stream(g + r, cg_);
                 ev[u] = load4_stream(e + r, ce);
             } else {
                 float gt[4], et[4];
@@ -100,13 +97,22 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t r = lane_r(r0, warp, half * 4 + u, lane);
+        for (int u = 0; u < 2; ++u) {
+            const int r = lane_r(r0, warp, bt * 2 + u, lane);
             float xs[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 xs[k] = __fadd_rn(lane_elem(gv[u], k), lane_elem(ev[u], k));  // line 7: x = g + e
-                if (FULL || r + k < len) atomicAdd(&sh[mag_key(xs[k]) >> 20], 1u);
+                if ((FULL || r + k < len) && mag_key(xs[k]) >= tau_hat) {
+                    const uint2 cv = make_uint2(coord0 + (uint32_t)(r + k), __float_as_uint(xs[k]));
+                    const uint32_t slot = atomicAdd(sh_cnt, 1u);
+                    if (slot < (uint32_t)kTileCand) {
+                        sh_cand[slot] = cv;
+                    } else {  // a tile dense with candidates: the staging buffer is full, append directly
+                        const uint32_t p = atomicAdd(g_cnt, 1u);
+                        if (p < cap) g_out[p] = cv;
+                    }
+                }
             }
             if (FULL || r + 3 < len) {
                 store4(e + r, ce, make_float4(xs[0], xs[1], xs[2], xs[3]));
@@ -119,39 +125,406 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
     }
 }
 
-__global__ void __launch_bounds__(kThreads) topk_sweep_kernel(Tables t, TopkBuffers b, const float* __restrict__ G) {
-    __shared__ uint32_t sh[kBins1];
-    const TileCoord c = tile_coord(t, blockIdx.y, blockIdx.x);
+__global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const float* __restrict__ G) {
+    __shared__ uint2 sh_cand[kTileCand];
+    __shared__ uint32_t sh_cnt, sh_base;
+    const TileInfo ti = load_tile(t.tiles, blockIdx.x);
+    const int i = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int k = threadIdx.x; k < kBins1; k += kThreads) sh[k] = 0u;
+    const size_t sg = (size_t)i * t.nseg + ti.seg;
+    SegState* st = b.seg + sg;
+    const uint32_t tau_hat = st->tau_hat;
+    const SegInfo* si = t.segs + ti.seg;
+    const uint32_t cap = si->cap;
+    uint2* out = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
+    if (threadIdx.x == 0) sh_cnt = 0u;
     __syncthreads();
-    const float* g = G + (size_t)c.i * (size_t)t.d + (size_t)c.o;
-    float* e = b.E + (size_t)c.i * (size_t)t.d + (size_t)c.o;
-    if (c.r0 + kTile <= c.len)
-        topk_sweep_tile<true>(g, e, c.len, c.r0, warp, lane, sh);
+    const float* g = G + (size_t)i * (size_t)t.d + (size_t)ti.o;
+    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
+    if (ti.r0 + kTile <= ti.len)
+        topk_sweep_tile<true>(g, e, ti.len, ti.r0, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
+                              &st->cand_count, out, cap);
     else
-        topk_sweep_tile<false>(g, e, c.len, c.r0, warp, lane, sh);
+        topk_sweep_tile<false>(g, e, ti.len, ti.r0, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
+                               &st->cand_count, out, cap);
     __syncthreads();
-    uint32_t* h = b.hist + c.sg * kBins1;
-    for (int k = threadIdx.x; k < kBins1; k += kThreads) {
-        uint32_t v = sh[k];
-        if (v) atomicAdd(h + k, v);
+    const uint32_t cnt = sh_cnt;
+    if (cnt == 0u) return;
+    const uint32_t stored = cnt < (uint32_t)kTileCand ? cnt : (uint32_t)kTileCand;
+    if (threadIdx.x == 0) sh_base = atomicAdd(&st->cand_count, stored);
+    __syncthreads();
+    const uint32_t base = sh_base;
+    for (uint32_t k = threadIdx.x; k < stored; k += kThreads)
+        if (base + k < cap) out[base + k] = sh_cand[k];
+}
+
+// ------------------------------------------------------------------------------------------
+// select: exact Top-k inside the candidate list, one CTA or one cluster of CTAs per segment
+
+// Prediction for the next step's sweep, from this step's threshold key `tau` and the bin edge
+// `edge` at or above which about 2.5 k_b keys lay: the threshold keeps rising while the error
+// accumulators fill, so tau_hat follows half of the last rise. `sel_shift` sizes the bins of the
+// next select so that the expected threshold lands near the middle of its 4096 bins.
+__device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_t edge, bool enabled) {
+    const uint32_t prev = st->tau_prev;
+    uint32_t rise = 0;
+    if (prev != kNoPrediction && tau > prev) rise = (tau - prev) >> 1;
+    if (edge > tau) edge = tau;
+    uint32_t next = edge + rise;
+    if (next >= 0x7f800000u) next = edge;
+    const uint32_t tau_pred = tau + rise;
+    uint32_t span = tau_pred > next ? tau_pred - next : 1u;
+    if (span < 2048u) span = 2048u;
+    st->sel_shift = 32u - (uint32_t)__clz(span >> 11);  // smallest S with span >> S < 2048
+    st->tau_hat = enabled ? next : kNoPrediction;
+    st->tau_prev = tau;
+}
+
+constexpr int kSurvCap = 1536;  // threshold-bin candidates one CTA can keep in shared memory
+constexpr int kSelUnroll = 8;   // candidate loads in flight per thread while scanning a list
+
+// Adds the `pred` lanes of a warp to a shared counter with one atomic; returns this lane's slot.
+__device__ __forceinline__ uint32_t warp_slot(bool pred, uint32_t* counter, int lane) {
+    const unsigned m = __ballot_sync(0xffffffffu, pred);
+    uint32_t base = 0;
+    if (m) {
+        const int leader = __ffs(m) - 1;
+        if (lane == leader) base = atomicAdd(counter, (uint32_t)__popc(m));
+        base = __shfl_sync(0xffffffffu, base, leader);
+    }
+    return base + (uint32_t)__popc(m & ((1u << lane) - 1u));
+}
+
+// A histogram of nb bins scanned from its top bin down: every thread owns nb / kThreads
+// consecutive bins (from the top) and learns how many entries lie above and inside its bins.
+struct BinScan {
+    uint32_t incl, excl;
+};
+__device__ __forceinline__ BinScan scan_from_top(const uint32_t* hm, int nb, uint32_t* scratch, uint32_t* total) {
+    const int per = nb / kThreads > 0 ? nb / kThreads : 1;
+    uint32_t sum = 0;
+    for (int j = 0; j < per; ++j) {
+        const int bin = nb - 1 - ((int)threadIdx.x * per + j);
+        if (bin >= 0) sum += hm[bin];
+    }
+    BinScan r;
+    r.incl = block_inclusive_scan(sum, scratch, total);
+    r.excl = r.incl - sum;
+    return r;
+}
+// The thread whose bins hold the `target`-th entry from the top writes
+// sh_out[0] = bin, sh_out[1] = entries above the bin, sh_out[2] = entries in the bin.
+__device__ __forceinline__ void locate(const uint32_t* hm, int nb, const BinScan& sc, uint32_t target, uint32_t* sh_out) {
+    if (sc.excl < target && target <= sc.incl) {
+        const int per = nb / kThreads > 0 ? nb / kThreads : 1;
+        uint32_t running = sc.excl;
+        for (int j = 0; j < per; ++j) {
+            const int bin = nb - 1 - ((int)threadIdx.x * per + j);
+            const uint32_t cj = bin >= 0 ? hm[bin] : 0u;
+            if (running < target && target <= running + cj) {
+                sh_out[0] = (uint32_t)bin;
+                sh_out[1] = running;
+                sh_out[2] = cj;
+            }
+            running += cj;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
+                                                               int nlist) {
+    __shared__ uint32_t local[kSelBins];   // this CTA's histogram
+    __shared__ uint32_t merged[kSelBins];  // rank 0's copy receives every CTA's counts
+    __shared__ uint2 surv[kSurvCap];
+    __shared__ uint32_t scratch[kWarps];
+    __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt, sh_ovf;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
+    const unsigned nrank = cluster.num_blocks();
+    const int lane = threadIdx.x & 31;
+    const size_t item = blockIdx.x / nrank;
+    const int i = (int)(item / (size_t)nlist);
+    const int seg = seg_list[item % (size_t)nlist];
+    const size_t sg = (size_t)i * t.nseg + seg;
+    const SegInfo* si = t.segs + seg;
+    SegState* st = b.seg + sg;
+    const uint32_t kb = si->kb, cap = si->cap;
+    const uint32_t c = st->cand_count;
+    const uint32_t tau_hat = st->tau_hat;
+    const int S = (int)st->sel_shift;
+    // the same decision in every CTA of the cluster: they read the same words and nobody writes them here
+    if (!(tau_hat != kNoPrediction && c >= kb && c <= cap)) {
+        if (rank == 0 && threadIdx.x == 0) {
+            st->fallback = 1u;
+            atomicAdd(b.dense_count, 1u);
+        }
+        return;
+    }
+    uint32_t* merged0 = cluster.map_shared_rank(&merged[0], 0);
+    uint32_t* ovf0 = cluster.map_shared_rank(&sh_ovf, 0);
+    const uint2* list = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
+    const uint32_t per = (c + nrank - 1) / nrank;
+    const uint32_t lo = rank * per;
+    const uint32_t hi = (lo + per < c) ? lo + per : c;
+    auto digit0 = [&](uint32_t xbits) -> uint32_t {
+        const uint32_t o = (xbits & 0x7fffffffu) - tau_hat;  // every candidate has key >= tau_hat
+        const uint32_t dg = o >> S;
+        return dg < (uint32_t)(kSelBins - 1) ? dg : (uint32_t)(kSelBins - 1);
+    };
+
+    // ---- pass 0: histogram of the key offsets above tau_hat in bins of 2^S; the last bin is open-ended
+    for (int k = threadIdx.x; k < kSelBins; k += kThreads) {
+        local[k] = 0u;
+        merged[k] = 0u;
+    }
+    if (threadIdx.x == 0) sh_ovf = 0u;
+    cluster.sync();
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+        uint32_t y[kSelUnroll];
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const uint32_t p = p0 + u * kThreads + threadIdx.x;
+            y[u] = p < hi ? list[p].y : 0xffffffffu;  // no candidate has this pattern (NaN)
+        }
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const bool valid = y[u] != 0xffffffffu;
+            const uint32_t dg = valid ? digit0(y[u]) : 0u;
+            // the open-ended last bin collects every far-above-threshold candidate: one atomic per warp
+            const bool far = valid && dg == (uint32_t)(kSelBins - 1);
+            const unsigned m = __ballot_sync(0xffffffffu, far);
+            if (m && lane == __ffs(m) - 1) atomicAdd(&local[kSelBins - 1], (uint32_t)__popc(m));
+            if (valid && !far) atomicAdd(&local[dg], 1u);
+        }
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < kSelBins; k += kThreads) {
+        const uint32_t v = local[k];
+        if (v) atomicAdd(merged0 + k, v);
+    }
+    cluster.sync();
+    uint32_t total;
+    {
+        const BinScan sc = scan_from_top(merged0, kSelBins, scratch, &total);
+        const uint32_t want = 2u * kb + (kb >> 1);
+        if (threadIdx.x == 0) sh_edge[0] = 0xffffffffu;  // "fewer than `want` candidates"
+        __syncthreads();
+        locate(merged0, kSelBins, sc, kb, sh_bin);
+        locate(merged0, kSelBins, sc, want, sh_edge);
+    }
+    __syncthreads();
+    const uint32_t b0 = sh_bin[0];
+    uint32_t k_rem = kb - sh_bin[1];
+    const uint32_t c0 = sh_bin[2];
+    const uint32_t edge_bin = sh_edge[0];
+    const bool take_all0 = (c0 == k_rem);
+    // this CTA's own share of the winners, from its private histogram
+    uint32_t mine = 0;
+    for (int k = threadIdx.x; k < kSelBins; k += kThreads)
+        if ((uint32_t)k > b0 || (take_all0 && (uint32_t)k == b0)) mine += local[k];
+    uint32_t my_winners;
+    block_inclusive_scan(mine, scratch, &my_winners);
+    cluster.sync();  // everybody has read rank 0's histogram
+    if (b0 == (uint32_t)(kSelBins - 1) && !take_all0) {
+        // the threshold lies in the open-ended bin: the prediction was far off, let the dense passes decide
+        if (rank == 0 && threadIdx.x == 0) {
+            st->fallback = 1u;
+            atomicAdd(b.dense_count, 1u);
+        }
+        return;
+    }
+
+    // ---- second scan of the list: winners to the message, threshold-bin candidates to shared memory
+    const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
+    if (threadIdx.x == 0) {
+        sh_base = my_winners ? atomicAdd(&st->emit_count, my_winners) : 0u;
+        sh_wcnt = 0u;
+        sh_scnt = 0u;
+    }
+    __syncthreads();
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+        uint2 cvs[kSelUnroll];
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const uint32_t p = p0 + u * kThreads + threadIdx.x;
+            cvs[u] = p < hi ? list[p] : make_uint2(0u, 0xffffffffu);
+        }
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const uint2 cv = cvs[u];
+            const bool valid = cv.y != 0xffffffffu;
+            const uint32_t dg = valid ? digit0(cv.y) : 0u;
+            const bool win = valid && (dg > b0 || (take_all0 && dg == b0));
+            const bool keep = valid && !take_all0 && dg == b0;
+            const uint32_t wpos = sh_base + warp_slot(win, &sh_wcnt, lane);
+            const uint32_t spos = warp_slot(keep, &sh_scnt, lane);
+            if (win) {
+                if (wpos < kb) {
+                    b.idx[slot0 + wpos] = (int32_t)cv.x;
+                    b.val[slot0 + wpos] = __uint_as_float(cv.y);
+                } else {
+                    atomicOr(b.status, 1u);
+                }
+            }
+            if (keep && spos < (uint32_t)kSurvCap) surv[spos] = cv;
+        }
+    }
+    __syncthreads();
+    // threshold key of this step (a lower bound if the select stops early)
+    const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
+    uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
+    if (!take_all0) {
+        const uint32_t nsurv = sh_scnt;
+        if (nsurv > (uint32_t)kSurvCap) atomicOr(ovf0, 1u);
+        cluster.sync();
+        const bool ovf = *ovf0 != 0u;
+        cluster.sync();  // rank 0 may leave only after everybody has read its flag
+        if (ovf) {
+            // too many candidates share the threshold bin (heavily duplicated values): dense passes
+            if (rank == 0 && threadIdx.x == 0) {
+                st->fallback = 1u;
+                atomicAdd(b.dense_count, 1u);
+            }
+            return;
+        }
+        // ---- radix select among the survivors over (low S key bits, ~index), 11 bits at a time
+        const uint32_t lowmask = S ? ((1u << S) - 1u) : 0u;
+        auto comp_of = [&](const uint2& cv) -> unsigned long long {
+            const uint32_t o = (cv.y & 0x7fffffffu) - tau_hat;
+            return ((unsigned long long)(o & lowmask) << 32) | (unsigned long long)(0xffffffffu - cv.x);
+        };
+        int top = S + 32;  // bits of the composite still undecided
+        unsigned long long prefix = 0ull;
+        bool take_all = false;
+#pragma unroll 1
+        while (top > 0 && !take_all) {
+            const int width = top < 11 ? top : 11;
+            const int shift = top - width;
+            const int nb = 1 << width;
+            for (int k = threadIdx.x; k < nb; k += kThreads) {
+                local[k] = 0u;
+                merged[k] = 0u;
+            }
+            cluster.sync();
+            for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
+                const unsigned long long cm = comp_of(surv[q]);
+                if ((cm >> top) == prefix) atomicAdd(&local[(uint32_t)(cm >> shift) & (uint32_t)(nb - 1)], 1u);
+            }
+            __syncthreads();
+            for (int k = threadIdx.x; k < nb; k += kThreads) {
+                const uint32_t v = local[k];
+                if (v) atomicAdd(merged0 + k, v);
+            }
+            cluster.sync();
+            {
+                uint32_t tot2;
+                const BinScan sc = scan_from_top(merged0, nb, scratch, &tot2);
+                locate(merged0, nb, sc, k_rem, sh_bin);
+            }
+            __syncthreads();
+            prefix = (prefix << width) | (unsigned long long)sh_bin[0];
+            k_rem -= sh_bin[1];
+            take_all = (sh_bin[2] == k_rem);
+            top = shift;
+            cluster.sync();  // rank 0's histogram has been read by everybody before it is cleared again
+        }
+        // kept survivors: composite >> top >= prefix
+        uint32_t cnt = 0;
+        for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) cnt += ((comp_of(surv[q]) >> top) >= prefix) ? 1u : 0u;
+        uint32_t tot3;
+        const uint32_t incl = block_inclusive_scan(cnt, scratch, &tot3);
+        if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
+        __syncthreads();
+        uint32_t pos = sh_base + incl - cnt;
+        for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
+            const uint2 cv = surv[q];
+            if ((comp_of(cv) >> top) >= prefix) {
+                if (pos < kb) {
+                    b.idx[slot0 + pos] = (int32_t)cv.x;
+                    b.val[slot0 + pos] = __uint_as_float(cv.y);
+                } else {
+                    atomicOr(b.status, 1u);
+                }
+                ++pos;
+            }
+        }
+        // decided low key bits of the threshold
+        const unsigned long long lowbits = top >= 32 ? (prefix << (top - 32)) : (prefix >> (32 - top));
+        tau += (uint32_t)lowbits & lowmask;
+    }
+    if (rank == 0 && threadIdx.x == 0) {
+        uint32_t edge;
+        if (edge_bin != 0xffffffffu) {
+            const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
+            edge = ew < 0x7f7fffffull ? (uint32_t)ew : 0x7f7fffffu;
+        } else {
+            // fewer than 2.5 k_b candidates: reach further down next time, by half the distance to the threshold
+            const uint32_t gap = ((tau - tau_hat) >> 1) + (1u << 16);
+            edge = tau_hat > gap ? tau_hat - gap : 0u;
+        }
+        predict_next(st, tau, edge, true);
+        st->fallback = 0u;
+        atomicAdd(b.status + 2, 1u);  // selections decided inside their candidate list
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// find: locate the bin that holds the k_rem-th largest key of a pass
+// dense passes, only for segments marked `fallback`
+
+template <int PASS>
+__global__ void __launch_bounds__(kThreads) topk_hist_kernel(Tables t, TopkBuffers b) {
+    constexpr int NB = (PASS == 1) ? kBins1 : kBins23;
+    __shared__ uint32_t sh[NB];
+    if (*b.dense_count == 0u) return;  // every segment was decided inside its candidate list
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t total = (int64_t)t.n * t.ntiles;
+    for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
+        const int i = (int)(w / t.ntiles);
+        const TileInfo ti = load_tile(t.tiles, (int)(w % t.ntiles));
+        const size_t sg = (size_t)i * t.nseg + ti.seg;
+        if (b.seg[sg].fallback == 0u) continue;
+        const uint32_t prefix = b.seg[sg].prefix;
+        for (int k = threadIdx.x; k < NB; k += kThreads) sh[k] = 0u;
+        __syncthreads();
+        const float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
+        float4 xv[kIters];
+        load_x_tile(e, ti.len, ti.r0, warp, lane, xv);
+        int any = 0;
+#pragma unroll
+        for (int it = 0; it < kIters; ++it) {
+            const int r = lane_r(ti.r0, warp, it, lane);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t key = mag_key(lane_elem(xv[it], k));
+                const bool match = (PASS == 1) ? true : (PASS == 2) ? ((key >> 20) == prefix) : ((key >> 10) == prefix);
+                if (match && r + k < ti.len) {
+                    atomicAdd(&sh[(PASS == 1) ? (key >> 20) : (PASS == 2) ? ((key >> 10) & 1023u) : (key & 1023u)], 1u);
+                    any = 1;
+                }
+            }
+        }
+        if (__syncthreads_or(any)) {
+            uint32_t* h = b.hist + sg * kBins1;
+            for (int k = threadIdx.x; k < NB; k += kThreads) {
+                const uint32_t v = sh[k];
+                if (v) atomicAdd(h + k, v);
+            }
+        }
+        __syncthreads();
+    }
+}
 
 template <int NBINS, int BITS, int PASS>
 __global__ void __launch_bounds__(kThreads) topk_find_kernel(Tables t, TopkBuffers b) {
     __shared__ uint32_t scratch[kWarps];
     constexpr int PER = NBINS / kThreads;
+    if (*b.dense_count == 0u) return;
     const size_t sg = blockIdx.x;
-    const int seg = (int)(sg % (size_t)t.nseg);
-    const int blk = t.tile_blk[t.seg_tile0[seg]];
     SegState* st = b.seg + sg;
+    if (st->fallback == 0u) return;
+    const SegInfo* si = t.segs + (sg % (size_t)t.nseg);
     uint32_t* h = b.hist + sg * kBins1;
-    const uint32_t kb = (uint32_t)(b.seg_off[blk + 1] - b.seg_off[blk]);
+    const uint32_t kb = si->kb;
     const uint32_t k_rem = (PASS == 1) ? kb : st->k_rem;
     const uint32_t prefix = (PASS == 1) ? 0u : st->prefix;
     // thread t owns the PER bins NBINS-1-t*PER ... downwards, so a scan over threads runs from the top bin down
@@ -182,80 +555,60 @@ __global__ void __launch_bounds__(kThreads) topk_find_kernel(Tables t, TopkBuffe
                     st->ties_total = cnt[j];
                     st->ties_take = nk;
                     st->need_order = (nk < cnt[j]) ? 1u : 0u;
-                    st->emit_count = 0u;
+                    // prediction for the next step's sweep (blocks without a candidate buffer never predict)
+                    predict_next(st, np, st->edge, si->cap != 0u);
                 }
             }
             running += cnt[j];
         }
     }
+    if (PASS == 1) {
+        // the highest pass-1 bin edge at or above which at least 2.5 k_b keys lie (0 if there are fewer);
+        // a candidate path that gave up may have handed out message slots: start over
+        const uint32_t want = 2u * kb + (kb >> 1);
+        if (threadIdx.x == 0) {
+            st->emit_count = 0u;
+            if (total < want) st->edge = 0u;
+        }
+        if (excl < want && want <= incl) {
+            uint32_t running = excl;
+#pragma unroll
+            for (int j = 0; j < PER; ++j) {
+                if (running < want && want <= running + cnt[j])
+                    st->edge = (uint32_t)(NBINS - 1 - ((int)threadIdx.x * PER + j)) << 20;
+                running += cnt[j];
+            }
+        }
+    }
     if (threadIdx.x == 0 && total < k_rem) atomicOr(b.status, 2u);
 }
-
-// ------------------------------------------------------------------------------------------
-// hist: passes 2 and 3 over x (read back from E), restricted to keys that match the prefix
-
-template <int PASS>
-__global__ void __launch_bounds__(kThreads) topk_hist_kernel(Tables t, TopkBuffers b) {
-    __shared__ uint32_t sh[kBins23];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t total = (int64_t)t.n * t.ntiles;
-    for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
-        const TileCoord c = tile_coord(t, (int)(w / t.ntiles), (int)(w % t.ntiles));
-        const uint32_t prefix = b.seg[c.sg].prefix;
-        for (int k = threadIdx.x; k < kBins23; k += kThreads) sh[k] = 0u;
-        __syncthreads();
-        const float* e = b.E + (size_t)c.i * (size_t)t.d + (size_t)c.o;
-        float4 xv[kIters];
-        load_x_tile(e, c.len, c.r0, warp, lane, xv);
-        int any = 0;
-#pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            const int64_t r = lane_r(c.r0, warp, it, lane);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const uint32_t key = mag_key(lane_elem(xv[it], k));
-                const bool match = (PASS == 2) ? ((key >> 20) == prefix) : ((key >> 10) == prefix);
-                if (match && r + k < c.len) {
-                    atomicAdd(&sh[(PASS == 2) ? ((key >> 10) & 1023u) : (key & 1023u)], 1u);
-                    any = 1;
-                }
-            }
-        }
-        if (__syncthreads_or(any)) {
-            uint32_t* h = b.hist + c.sg * kBins1;
-            for (int k = threadIdx.x; k < kBins23; k += kThreads) {
-                uint32_t v = sh[k];
-                if (v) atomicAdd(h + k, v);
-            }
-        }
-        __syncthreads();
-    }
-}
-
-// ------------------------------------------------------------------------------------------
-// collect: emit everything above the threshold (and the ties when all of them fit)
 
 __global__ void __launch_bounds__(kThreads) topk_collect_kernel(Tables t, TopkBuffers b) {
     __shared__ uint32_t scratch[kWarps];
     __shared__ uint32_t sh_base;
+    if (*b.dense_count == 0u) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t total = (int64_t)t.n * t.ntiles;
     for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
-        const TileCoord c = tile_coord(t, (int)(w / t.ntiles), (int)(w % t.ntiles));
-        SegState* st = b.seg + c.sg;
+        const int i = (int)(w / t.ntiles);
+        const int tile = (int)(w % t.ntiles);
+        const TileInfo ti = load_tile(t.tiles, tile);
+        const size_t sg = (size_t)i * t.nseg + ti.seg;
+        SegState* st = b.seg + sg;
+        if (st->fallback == 0u) continue;
         const uint32_t tau = st->tau;
         const bool need_order = st->need_order != 0u;
-        float* e = b.E + (size_t)c.i * (size_t)t.d + (size_t)c.o;
+        const float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
         float4 xv[kIters];
-        load_x_tile(e, c.len, c.r0, warp, lane, xv);
+        load_x_tile(e, ti.len, ti.r0, warp, lane, xv);
         uint32_t n_emit = 0, n_tie = 0;
 #pragma unroll
         for (int it = 0; it < kIters; ++it) {
-            const int64_t r = lane_r(c.r0, warp, it, lane);
+            const int r = lane_r(ti.r0, warp, it, lane);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const uint32_t key = mag_key(lane_elem(xv[it], k));
-                const bool live = r + k < c.len;
+                const bool live = r + k < ti.len;
                 n_emit += (live && key > tau) ? 1u : 0u;
                 n_tie += (live && key == tau) ? 1u : 0u;
             }
@@ -265,25 +618,26 @@ __global__ void __launch_bounds__(kThreads) topk_collect_kernel(Tables t, TopkBu
         const uint32_t incl = block_inclusive_scan(n_emit, scratch, &tot);
         if (need_order) {
             block_inclusive_scan(n_tie, scratch, &tie_tot);
-            if (threadIdx.x == 0) b.tile_ties[(size_t)c.i * t.ntiles + c.tile] = tie_tot;
+            if (threadIdx.x == 0) b.tile_ties[(size_t)i * t.ntiles + tile] = tie_tot;
         }
         if (tot) {
             if (threadIdx.x == 0) sh_base = atomicAdd(&st->emit_count, tot);
             __syncthreads();
-            const uint32_t kb = (uint32_t)(b.seg_off[c.blk + 1] - b.seg_off[c.blk]);
-            const size_t slot0 = (size_t)c.i * (size_t)b.K + (size_t)b.seg_off[c.blk];
+            const SegInfo* si = t.segs + ti.seg;
+            const uint32_t kb = si->kb;
+            const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
             uint32_t pos = sh_base + (incl - n_emit);
 #pragma unroll
             for (int it = 0; it < kIters; ++it) {
-                const int64_t r = lane_r(c.r0, warp, it, lane);
+                const int r = lane_r(ti.r0, warp, it, lane);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const float x = lane_elem(xv[it], k);
                     const uint32_t key = mag_key(x);
-                    const bool live = r + k < c.len;
+                    const bool live = r + k < ti.len;
                     if (live && (key > tau || (!need_order && key == tau))) {
                         if (pos < kb) {
-                            b.idx[slot0 + pos] = (int32_t)(c.o + r + k);
+                            b.idx[slot0 + pos] = (int32_t)(ti.o + r + k);
                             b.val[slot0 + pos] = x;
                         } else {
                             atomicOr(b.status, 1u);
@@ -297,34 +651,37 @@ __global__ void __launch_bounds__(kThreads) topk_collect_kernel(Tables t, TopkBu
     }
 }
 
-// ------------------------------------------------------------------------------------------
-// ties: when only some of the keys equal to the threshold fit, take those with the lowest index
-
+// Closes the step for one segment: if the dense passes left threshold ties to order, takes those
+// with the lowest index; then checks that exactly k_b entries were emitted and resets the counters.
 __global__ void __launch_bounds__(kThreads) topk_ties_kernel(Tables t, TopkBuffers b) {
     __shared__ uint32_t scratch[kWarps];
     __shared__ uint32_t sh_c[kThreads], sh_excl[kThreads];
     const size_t sg = blockIdx.x;
     const int i = (int)(sg / (size_t)t.nseg);
-    const int seg = (int)(sg % (size_t)t.nseg);
-    const int tile0 = t.seg_tile0[seg], tile_end = t.seg_tile0[seg + 1];
-    const int blk = t.tile_blk[tile0];
+    const SegInfo* si = t.segs + (sg % (size_t)t.nseg);
     SegState* st = b.seg + sg;
-    const uint32_t kb = (uint32_t)(b.seg_off[blk + 1] - b.seg_off[blk]);
+    const uint32_t kb = si->kb;
     const uint32_t emitted = st->emit_count;
-    if (!st->need_order) {
-        if (threadIdx.x == 0 && emitted != kb) atomicOr(b.status, 1u);
-        return;
-    }
+    const bool dense = st->fallback != 0u;
+    const bool need_order = dense && st->need_order != 0u;
     const uint32_t tau = st->tau;
-    const uint32_t want = st->ties_take;
-    if (emitted + want != kb) {
-        if (threadIdx.x == 0) atomicOr(b.status, 1u);
-        return;
+    const uint32_t want = need_order ? st->ties_take : 0u;
+    __syncthreads();  // every thread has read the state before thread 0 resets it
+    if (threadIdx.x == 0) {
+        if (emitted + want != kb) atomicOr(b.status, 1u);
+        if (dense) atomicAdd(b.status + 1, 1u);              // selections decided by the dense passes
+        if (dense && si->cap) atomicSub(b.dense_count, 1u);  // back to the number of blocks that never predict
+        st->emit_count = 0u;
+        st->cand_count = 0u;
+        st->fallback = si->cap ? 0u : 1u;  // blocks without a candidate buffer always take the dense passes
+        st->need_order = 0u;
     }
-    const int64_t o = t.off[blk];
-    const int64_t len = t.off[blk + 1] - o;
-    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
-    const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)b.seg_off[blk];
+    if (!need_order || emitted + want != kb) return;
+    const int tile0 = si->tile0, tile_end = si->tile0 + si->ntile_b;
+    const int64_t o = si->o;
+    const int len = si->len;
+    const float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
+    const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
     uint32_t taken = 0;  // ties already assigned to earlier tiles (uniform across the CTA)
     for (int tb = tile0; tb < tile_end && taken < want; tb += kThreads) {
         const int tt = tb + (int)threadIdx.x;
@@ -342,20 +699,18 @@ __global__ void __launch_bounds__(kThreads) topk_ties_kernel(Tables t, TopkBuffe
             if (before >= want) break;
             const uint32_t take = (cq < want - before) ? cq : want - before;
             // tile tb+q in index order: thread j owns the 32 consecutive coordinates r0 + 32 j ...
-            const int64_t r0 = t.tile_r0[tb + q];
-            const int64_t rs = r0 + (int64_t)threadIdx.x * 32;
+            const int rs = (tb + q - tile0) * kTile + (int)threadIdx.x * 32;
             uint32_t mine = 0;
             for (int k = 0; k < 32; ++k) {
-                const int64_t r = rs + k;
+                const int r = rs + k;
                 if (r < len && mag_key(e[r]) == tau) mine |= 1u << k;
             }
             uint32_t tile_tot;
-            const uint32_t rank0 = block_inclusive_scan((uint32_t)__popc(mine), scratch, &tile_tot) - __popc(mine);
-            uint32_t rank = rank0;
+            uint32_t rank = block_inclusive_scan((uint32_t)__popc(mine), scratch, &tile_tot) - __popc(mine);
             while (mine && rank < take) {
                 const int k = __ffs(mine) - 1;
                 mine &= mine - 1;
-                const int64_t r = rs + k;
+                const int r = rs + k;
                 const uint32_t pos = emitted + before + rank;
                 if (pos < kb) {
                     b.idx[slot0 + pos] = (int32_t)(o + r);
@@ -390,7 +745,7 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 
     // radix select over the 31-bit key: digits of 8, 8, 8 and 7 bits from the top
     uint32_t prefix = 0, k_rem = kb;
-    int shift = 31;       // bits below `shift` are still undecided
+    int shift = 31;         // bits below `shift` are still undecided
     bool take_all = false;  // every key in the chosen bin is kept: no tie to break
 #pragma unroll 1
     for (int pass = 0; pass < 4 && !take_all; ++pass) {
@@ -503,6 +858,30 @@ cudaError_t launch_topk_sweep(compams_context* c, const float* grads) {
     return cudaGetLastError();
 }
 
+// One launch per list of segments: short candidate lists get one CTA each, long ones a cluster.
+static cudaError_t launch_select_list(compams_context* c, const int32_t* list, int nlist, int cluster) {
+    if (nlist == 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((int64_t)c->n * nlist * cluster), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, topk_select_kernel, c->tab, c->tk, list, nlist);
+}
+
+cudaError_t launch_topk_select(compams_context* c) {
+    cudaError_t e = launch_select_list(c, c->sel_small, c->n_sel_small, 1);
+    if (e != cudaSuccess) return e;
+    return launch_select_list(c, c->sel_big, c->n_sel_big, kSelectCluster);
+}
+
 cudaError_t launch_topk_find(compams_context* c, int pass) {
     const unsigned grid = (unsigned)((int64_t)c->n * c->tab.nseg);
     if (pass == 1)
@@ -516,7 +895,9 @@ cudaError_t launch_topk_find(compams_context* c, int pass) {
 
 cudaError_t launch_topk_hist(compams_context* c, int pass) {
     const int grid = persistent_grid(c, (int64_t)c->n * c->tab.ntiles, 8);
-    if (pass == 2)
+    if (pass == 1)
+        topk_hist_kernel<1><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
+    else if (pass == 2)
         topk_hist_kernel<2><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
     else
         topk_hist_kernel<3><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
