@@ -45,13 +45,13 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
             const int r = rw + (bt * 2 + u) * 128 + lane * 4;
             if (FULL || r + 3 < len) {
                 gv[u] = load4_stream(g + r, cg);
-                ev[u] = load4_stream(e + r, ce);
+                ev[u] = load4(e + r, ce);
             } else {
                 float gt[4], et[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    gt[k] = (r + k < len) ? __ldcs(g + r + k) : 0.0f;
-                    et[k] = (r + k < len) ? __ldcs(e + r + k) : 0.0f;
+                    gt[k] = (r + k < len) ? __ldg(g + r + k) : 0.0f;
+                    et[k] = (r + k < len) ? e[r + k] : 0.0f;
                 }
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
                 ev[u] = make_float4(et[0], et[1], et[2], et[3]);
@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(kThreads) bs_apply_kernel(Tables t, BsBuffers 
         const int nc = (t.n - i0 < kApplyChunk) ? t.n - i0 : kApplyChunk;
         __syncthreads();
         for (int c = 0; c < nc; ++c)
-            sh_bits[c][threadIdx.x] = word_live ? __ldcs(b.bits + (size_t)(i0 + c) * (size_t)b.W + wbase + threadIdx.x) : 0u;
+            sh_bits[c][threadIdx.x] = word_live ? __ldg(b.bits + (size_t)(i0 + c) * (size_t)b.W + wbase + threadIdx.x) : 0u;
         if (threadIdx.x < nc) sh_s[threadIdx.x] = (double)b.scales_cur[(size_t)(i0 + threadIdx.x) * t.M + blk];
         __syncthreads();
         for (int c = 0; c < nc; ++c) {
@@ -205,8 +205,7 @@ __global__ void __launch_bounds__(kThreads) bs_apply_kernel(Tables t, BsBuffers 
 #pragma unroll
         for (int k = 0; k < 4; ++k) gb[k] = mean_from_acc(acc[it][k], hp.nf);
         if (r + 3 < len) {
-            float4 mm = load4_stream(m + r, cls), vv = load4_stream(v + r, cls), hh = load4_stream(vh + r, cls),
-                   tt = load4_stream(th + r, cls);
+            float4 mm = load4(m + r, cls), vv = load4(v + r, cls), hh = load4(vh + r, cls), tt = load4(th + r, cls);
             amsgrad_update(gb[0], mm.x, vv.x, hh.x, tt.x, hp);
             amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);
             amsgrad_update(gb[2], mm.z, vv.z, hh.z, tt.z, hp);

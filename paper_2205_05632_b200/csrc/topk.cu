@@ -84,13 +84,13 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
             const int r = lane_r(r0, warp, bt * 2 + u, lane);
             if (FULL || r + 3 < len) {
                 gv[u] = load4_stream(g + r, cg_);
-                ev[u] = load4_stream(e + r, ce);
+                ev[u] = load4(e + r, ce);
             } else {
                 float gt[4], et[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    gt[k] = (r + k < len) ? __ldcs(g + r + k) : 0.0f;
-                    et[k] = (r + k < len) ? __ldcs(e + r + k) : 0.0f;
+                    gt[k] = (r + k < len) ? __ldg(g + r + k) : 0.0f;
+                    et[k] = (r + k < len) ? e[r + k] : 0.0f;
                 }
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
                 ev[u] = make_float4(et[0], et[1], et[2], et[3]);
@@ -741,7 +741,7 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
     const uint32_t kb = (uint32_t)(b.seg_off[blk + 1] - b.seg_off[blk]);
     const float* g = G + (size_t)i * (size_t)t.d + (size_t)o;
     float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
-    for (int r = threadIdx.x; r < len; r += kThreads) xs[r] = __float_as_uint(__fadd_rn(__ldcs(g + r), e[r]));
+    for (int r = threadIdx.x; r < len; r += kThreads) xs[r] = __float_as_uint(__fadd_rn(__ldg(g + r), e[r]));
 
     // radix select over the 31-bit key: digits of 8, 8, 8 and 7 bits from the top
     uint32_t prefix = 0, k_rem = kb;
