@@ -149,84 +149,75 @@ __global__ void __launch_bounds__(kThreads) bs_materialize_kernel(Tables t, floa
     }
 }
 
-constexpr int kApplyChunk = 32;  // workers whose sign words are staged in shared memory at a time
+constexpr int kApplyChunk = 64;  // workers whose sign words are staged in shared memory at a time
 
-__global__ void __launch_bounds__(kThreads) bs_apply_kernel(Tables t, BsBuffers b, float* __restrict__ theta,
-                                                            HyperParams hp) {
-    __shared__ uint32_t sh_bits[kApplyChunk][kTile / 32];
+// One CTA per 1024 consecutive coordinates of a block (one float4 group per thread).
+__global__ void __launch_bounds__(kThreads, 6) bs_apply_kernel(Tables t, BsBuffers b, float* __restrict__ theta,
+                                                               HyperParams hp) {
+    __shared__ uint32_t sh_bits[kApplyChunk][32];
     __shared__ double sh_s[kApplyChunk];
-    const TileInfo ti = load_tile(t.tiles, blockIdx.x);
+    const TileInfo ti = load_tile(t.tiles, blockIdx.x >> 3);
     const int blk = ti.blk;
-    const int64_t o = ti.o;
-    const int64_t len = ti.len;
-    const int64_t r0 = ti.r0;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t rw = r0 + (int64_t)warp * kWarpSpan;
+    const int len = ti.len;
+    const int rs = ti.r0 + (int)(blockIdx.x & 7) * kWarpSpan;  // first coordinate of this CTA, relative to the block
+    if (rs >= len) return;
+    const int r = rs + (int)threadIdx.x * 4;
+    const int wsel = threadIdx.x >> 3, nsh = (threadIdx.x & 7) * 4;
 
-    double acc[kIters][4];
-#pragma unroll
-    for (int it = 0; it < kIters; ++it)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[it][k] = 0.0;
-
-    const size_t wbase = (size_t)b.word_off[blk] + (size_t)(r0 >> 5);
-    const bool word_live = r0 + (int64_t)threadIdx.x * 32 < len;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    const size_t wbase = (size_t)b.word_off[blk] + (size_t)(rs >> 5);
+    const int wl = threadIdx.x & 31, wr = threadIdx.x >> 5;  // word and worker this thread stages
+    const bool word_live = rs + wl * 32 < len;
     for (int i0 = 0; i0 < t.n; i0 += kApplyChunk) {
         const int nc = (t.n - i0 < kApplyChunk) ? t.n - i0 : kApplyChunk;
         __syncthreads();
-        for (int c = 0; c < nc; ++c)
-            sh_bits[c][threadIdx.x] = word_live ? __ldg(b.bits + (size_t)(i0 + c) * (size_t)b.W + wbase + threadIdx.x) : 0u;
+        for (int c = wr; c < nc; c += kWarps)
+            sh_bits[c][wl] = word_live ? __ldg(b.bits + (size_t)(i0 + c) * (size_t)b.W + wbase + wl) : 0u;
         if (threadIdx.x < nc) sh_s[threadIdx.x] = (double)b.scales_cur[(size_t)(i0 + threadIdx.x) * t.M + blk];
         __syncthreads();
+#pragma unroll 4
         for (int c = 0; c < nc; ++c) {
             const double s = sh_s[c];
             const double ns = -s;
-#pragma unroll
-            for (int it = 0; it < kIters; ++it) {
-                const uint32_t w = sh_bits[c][warp * 32 + it * 4 + (lane >> 3)];
-                const uint32_t nib = w >> ((lane & 7) * 4);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) acc[it][k] += ((nib >> k) & 1u) ? ns : s;
-            }
+            const uint32_t nib = sh_bits[c][wsel] >> nsh;
+            a0 += (nib & 1u) ? ns : s;
+            a1 += (nib & 2u) ? ns : s;
+            a2 += (nib & 4u) ? ns : s;
+            a3 += (nib & 8u) ? ns : s;
         }
     }
-
+    if (r >= len) return;
+    const int64_t o = ti.o;
     float* gbar = b.gbar + o;
     float* m = b.m + o;
     float* v = b.v + o;
     float* vh = b.vhat + o;
     float* th = theta + o;
     const int cls = align_class(m);  // all five vectors are 16-byte aligned at coordinate 0
+    const float gb[4] = {mean_from_acc(a0, hp.nf), mean_from_acc(a1, hp.nf), mean_from_acc(a2, hp.nf),
+                         mean_from_acc(a3, hp.nf)};
+    if (r + 3 < len) {
+        float4 mm = load4(m + r, cls), vv = load4(v + r, cls), hh = load4(vh + r, cls), tt = load4(th + r, cls);
+        amsgrad_update(gb[0], mm.x, vv.x, hh.x, tt.x, hp);
+        amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);
+        amsgrad_update(gb[2], mm.z, vv.z, hh.z, tt.z, hp);
+        amsgrad_update(gb[3], mm.w, vv.w, hh.w, tt.w, hp);
+        store4(gbar + r, cls, make_float4(gb[0], gb[1], gb[2], gb[3]));
+        store4(m + r, cls, mm);
+        store4(v + r, cls, vv);
+        store4(vh + r, cls, hh);
+        store4(th + r, cls, tt);
+    } else {
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int64_t r = rw + it * 128 + lane * 4;
-        if (r >= len) continue;
-        float gb[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) gb[k] = mean_from_acc(acc[it][k], hp.nf);
-        if (r + 3 < len) {
-            float4 mm = load4(m + r, cls), vv = load4(v + r, cls), hh = load4(vh + r, cls), tt = load4(th + r, cls);
-            amsgrad_update(gb[0], mm.x, vv.x, hh.x, tt.x, hp);
-            amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);
-            amsgrad_update(gb[2], mm.z, vv.z, hh.z, tt.z, hp);
-            amsgrad_update(gb[3], mm.w, vv.w, hh.w, tt.w, hp);
-            store4(gbar + r, cls, make_float4(gb[0], gb[1], gb[2], gb[3]));
-            store4(m + r, cls, mm);
-            store4(v + r, cls, vv);
-            store4(vh + r, cls, hh);
-            store4(th + r, cls, tt);
-        } else {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                if (r + k < len) {
-                    float mm = m[r + k], vv = v[r + k], hh = vh[r + k], tt = th[r + k];
-                    amsgrad_update(gb[k], mm, vv, hh, tt, hp);
-                    gbar[r + k] = gb[k];
-                    m[r + k] = mm;
-                    v[r + k] = vv;
-                    vh[r + k] = hh;
-                    th[r + k] = tt;
-                }
+        for (int k = 0; k < 4; ++k) {
+            if (r + k < len) {
+                float mm = m[r + k], vv = v[r + k], hh = vh[r + k], tt = th[r + k];
+                amsgrad_update(gb[k], mm, vv, hh, tt, hp);
+                gbar[r + k] = gb[k];
+                m[r + k] = mm;
+                v[r + k] = vv;
+                vh[r + k] = hh;
+                th[r + k] = tt;
             }
         }
     }
@@ -252,7 +243,7 @@ cudaError_t launch_bs_scales(compams_context* c) {
 cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     BsBuffers b = c->bs;
     b.scales_cur = c->scales[c->scales_cur];
-    bs_apply_kernel<<<(unsigned)c->tab.ntiles, kThreads, 0, c->stream>>>(c->tab, b, theta, c->hp);
+    bs_apply_kernel<<<(unsigned)c->tab.ntiles * kWarps, kThreads, 0, c->stream>>>(c->tab, b, theta, c->hp);
     return cudaGetLastError();
 }
 

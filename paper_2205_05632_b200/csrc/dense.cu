@@ -11,17 +11,18 @@
 
 namespace compams {
 
-__global__ void __launch_bounds__(kThreads) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const float* __restrict__ G,
-                                                                      float* __restrict__ gbar, float* __restrict__ m,
-                                                                      float* __restrict__ v, float* __restrict__ vhat,
-                                                                      float* __restrict__ theta, HyperParams hp) {
+// One CTA per 1024 coordinates: one float4 group per thread, the workers' rows read one after another.
+__global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const float* __restrict__ G,
+                                                                         float* __restrict__ gbar, float* __restrict__ m,
+                                                                         float* __restrict__ v, float* __restrict__ vhat,
+                                                                         float* __restrict__ theta, HyperParams hp) {
     const int64_t groups = d >> 2;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < groups; q += stride) {
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < groups) {
         const int64_t j = q << 2;
         double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
         const float* p = G + j;
-#pragma unroll 8
+#pragma unroll 4
         for (int32_t i = 0; i < n; ++i) {
             const float* pi = p + (size_t)i * (size_t)d;
             float4 g = load4_stream(pi, align_class(pi));
@@ -112,7 +113,9 @@ static int grid_for(const compams_context* c, int64_t work_items, int ctas_per_s
 }
 
 cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, float* theta) {
-    int grid = grid_for(c, c->d >> 2, 8);
+    int64_t groups = c->d >> 2;
+    int grid = (int)((groups + kThreads - 1) / kThreads);
+    if (grid < 1) grid = 1;
     dense_mean_amsgrad_kernel<<<grid, kThreads, 0, c->stream>>>(c->n, c->d, grads, c->gbar, c->m, c->v, c->vhat, theta,
                                                                 c->hp);
     return cudaGetLastError();
