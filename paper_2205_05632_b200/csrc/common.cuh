@@ -128,7 +128,8 @@ __device__ __forceinline__ TileInfo load_tile(const TileInfo* tiles, int tile) {
 }
 
 // Inclusive scan of one unsigned value per thread across a CTA of kThreads threads.
-// `scratch` holds kWarps words. Returns the inclusive prefix; *total receives the CTA sum.
+// `scratch` holds NWARPS words (the CTA has NWARPS warps). Returns the inclusive prefix; *total receives the CTA sum.
+template <int NWARPS = kWarps>
 __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t x, uint32_t* scratch, uint32_t* total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t s = x;
@@ -142,7 +143,7 @@ __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t x, uint32_t* s
     __syncthreads();
     uint32_t base = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < NWARPS; ++w) {
         uint32_t c = scratch[w];
         if (w < warp) base += c;
         tot += c;

@@ -15,8 +15,8 @@
 //                   holds at least k_b and at most its capacity, the exact Top-k is inside it. A
 //                   histogram of the key offsets above tau_hat (bins sized from the last step, merged
 //                   through distributed shared memory) finds the threshold bin; winners above it are
-//                   emitted, the bin's few candidates go to shared memory and a radix select over
-//                   (low key bits, ~index) composites finishes the job and predicts the next tau_hat.
+//                   emitted, the bin's few candidates go to rank 0's shared memory, which orders them
+//                   by (key, lower index first), keeps the best and predicts the next tau_hat.
 //                   Otherwise the segment is marked for the dense passes.
 //   Dense passes (only for marked segments; exact for any input, e.g. all-equal values):
 //     topk_hist<1..3> / topk_find<1..3>  three histogram passes over x, 11 + 10 + 10 key bits
@@ -181,7 +181,9 @@ __device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_
 }
 
 constexpr int kSurvCap = 1536;  // threshold-bin candidates one CTA can keep in shared memory
-constexpr int kSelUnroll = 8;   // candidate loads in flight per thread while scanning a list
+constexpr int kSelUnroll = 4;   // candidate loads in flight per thread while scanning a list
+constexpr int kSelThreads = 1024;  // a select CTA is alone on its SM: many threads keep enough loads in flight
+constexpr int kSelWarps = kSelThreads / 32;
 
 // Adds the `pred` lanes of a warp to a shared counter with one atomic; returns this lane's slot.
 __device__ __forceinline__ uint32_t warp_slot(bool pred, uint32_t* counter, int lane) {
@@ -201,14 +203,14 @@ struct BinScan {
     uint32_t incl, excl;
 };
 __device__ __forceinline__ BinScan scan_from_top(const uint32_t* hm, int nb, uint32_t* scratch, uint32_t* total) {
-    const int per = nb / kThreads > 0 ? nb / kThreads : 1;
+    const int per = nb / kSelThreads > 0 ? nb / kSelThreads : 1;
     uint32_t sum = 0;
     for (int j = 0; j < per; ++j) {
         const int bin = nb - 1 - ((int)threadIdx.x * per + j);
         if (bin >= 0) sum += hm[bin];
     }
     BinScan r;
-    r.incl = block_inclusive_scan(sum, scratch, total);
+    r.incl = block_inclusive_scan<kSelWarps>(sum, scratch, total);
     r.excl = r.incl - sum;
     return r;
 }
@@ -216,7 +218,7 @@ __device__ __forceinline__ BinScan scan_from_top(const uint32_t* hm, int nb, uin
 // sh_out[0] = bin, sh_out[1] = entries above the bin, sh_out[2] = entries in the bin.
 __device__ __forceinline__ void locate(const uint32_t* hm, int nb, const BinScan& sc, uint32_t target, uint32_t* sh_out) {
     if (sc.excl < target && target <= sc.incl) {
-        const int per = nb / kThreads > 0 ? nb / kThreads : 1;
+        const int per = nb / kSelThreads > 0 ? nb / kSelThreads : 1;
         uint32_t running = sc.excl;
         for (int j = 0; j < per; ++j) {
             const int bin = nb - 1 - ((int)threadIdx.x * per + j);
@@ -231,13 +233,13 @@ __device__ __forceinline__ void locate(const uint32_t* hm, int nb, const BinScan
     }
 }
 
-__global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
+__global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                int nlist) {
     __shared__ uint32_t local[kSelBins];   // this CTA's histogram
     __shared__ uint32_t merged[kSelBins];  // rank 0's copy receives every CTA's counts
     __shared__ uint2 surv[kSurvCap];
-    __shared__ uint32_t scratch[kWarps];
-    __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt, sh_ovf;
+    __shared__ uint32_t scratch[kSelWarps];
+    __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt;
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned rank = cluster.block_rank();
     const unsigned nrank = cluster.num_blocks();
@@ -261,7 +263,6 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
         return;
     }
     uint32_t* merged0 = cluster.map_shared_rank(&merged[0], 0);
-    uint32_t* ovf0 = cluster.map_shared_rank(&sh_ovf, 0);
     const uint2* list = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
     const uint32_t per = (c + nrank - 1) / nrank;
     const uint32_t lo = rank * per;
@@ -273,17 +274,17 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
     };
 
     // ---- pass 0: histogram of the key offsets above tau_hat in bins of 2^S; the last bin is open-ended
-    for (int k = threadIdx.x; k < kSelBins; k += kThreads) {
+    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads) {
         local[k] = 0u;
         merged[k] = 0u;
     }
-    if (threadIdx.x == 0) sh_ovf = 0u;
+    if (threadIdx.x == 0) sh_scnt = 0u;
     cluster.sync();
-    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kSelThreads) {
         uint32_t y[kSelUnroll];
 #pragma unroll
         for (int u = 0; u < kSelUnroll; ++u) {
-            const uint32_t p = p0 + u * kThreads + threadIdx.x;
+            const uint32_t p = p0 + u * kSelThreads + threadIdx.x;
             y[u] = p < hi ? list[p].y : 0xffffffffu;  // no candidate has this pattern (NaN)
         }
 #pragma unroll
@@ -298,7 +299,7 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
         }
     }
     __syncthreads();
-    for (int k = threadIdx.x; k < kSelBins; k += kThreads) {
+    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads) {
         const uint32_t v = local[k];
         if (v) atomicAdd(merged0 + k, v);
     }
@@ -320,10 +321,10 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
     const bool take_all0 = (c0 == k_rem);
     // this CTA's own share of the winners, from its private histogram
     uint32_t mine = 0;
-    for (int k = threadIdx.x; k < kSelBins; k += kThreads)
+    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads)
         if ((uint32_t)k > b0 || (take_all0 && (uint32_t)k == b0)) mine += local[k];
     uint32_t my_winners;
-    block_inclusive_scan(mine, scratch, &my_winners);
+    block_inclusive_scan<kSelWarps>(mine, scratch, &my_winners);
     cluster.sync();  // everybody has read rank 0's histogram
     if (b0 == (uint32_t)(kSelBins - 1) && !take_all0) {
         // the threshold lies in the open-ended bin: the prediction was far off, let the dense passes decide
@@ -334,19 +335,20 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
         return;
     }
 
-    // ---- second scan of the list: winners to the message, threshold-bin candidates to shared memory
+    // ---- second scan of the list: winners to the message, threshold-bin candidates to rank 0's shared memory
     const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
+    uint2* surv0 = cluster.map_shared_rank(&surv[0], 0);
+    uint32_t* scnt0 = cluster.map_shared_rank(&sh_scnt, 0);
     if (threadIdx.x == 0) {
         sh_base = my_winners ? atomicAdd(&st->emit_count, my_winners) : 0u;
         sh_wcnt = 0u;
-        sh_scnt = 0u;
     }
     __syncthreads();
-    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kSelThreads) {
         uint2 cvs[kSelUnroll];
 #pragma unroll
         for (int u = 0; u < kSelUnroll; ++u) {
-            const uint32_t p = p0 + u * kThreads + threadIdx.x;
+            const uint32_t p = p0 + u * kSelThreads + threadIdx.x;
             cvs[u] = p < hi ? list[p] : make_uint2(0u, 0xffffffffu);
         }
 #pragma unroll
@@ -357,7 +359,6 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
             const bool win = valid && (dg > b0 || (take_all0 && dg == b0));
             const bool keep = valid && !take_all0 && dg == b0;
             const uint32_t wpos = sh_base + warp_slot(win, &sh_wcnt, lane);
-            const uint32_t spos = warp_slot(keep, &sh_scnt, lane);
             if (win) {
                 if (wpos < kb) {
                     b.idx[slot0 + wpos] = (int32_t)cv.x;
@@ -366,91 +367,62 @@ __global__ void __launch_bounds__(kThreads) topk_select_kernel(Tables t, TopkBuf
                     atomicOr(b.status, 1u);
                 }
             }
-            if (keep && spos < (uint32_t)kSurvCap) surv[spos] = cv;
+            if (__any_sync(0xffffffffu, keep)) {  // rare: only the threshold bin's candidates
+                const uint32_t spos = warp_slot(keep, scnt0, lane);
+                if (keep && spos < (uint32_t)kSurvCap) surv0[spos] = cv;
+            }
         }
     }
-    __syncthreads();
-    // threshold key of this step (a lower bound if the select stops early)
+    // threshold key of this step (a lower bound if every candidate of the threshold bin is kept)
     const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
     uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
     if (!take_all0) {
+        cluster.sync();  // every CTA's threshold-bin candidates have reached rank 0
+        if (rank != 0) return;
         const uint32_t nsurv = sh_scnt;
-        if (nsurv > (uint32_t)kSurvCap) atomicOr(ovf0, 1u);
-        cluster.sync();
-        const bool ovf = *ovf0 != 0u;
-        cluster.sync();  // rank 0 may leave only after everybody has read its flag
-        if (ovf) {
+        if (nsurv > (uint32_t)kSurvCap) {
             // too many candidates share the threshold bin (heavily duplicated values): dense passes
-            if (rank == 0 && threadIdx.x == 0) {
+            if (threadIdx.x == 0) {
                 st->fallback = 1u;
                 atomicAdd(b.dense_count, 1u);
             }
             return;
         }
-        // ---- radix select among the survivors over (low S key bits, ~index), 11 bits at a time
+        // ---- rank 0 orders the survivors by (key, lower index first): survivor q is kept when fewer
+        // than k_rem survivors beat it
         const uint32_t lowmask = S ? ((1u << S) - 1u) : 0u;
         auto comp_of = [&](const uint2& cv) -> unsigned long long {
             const uint32_t o = (cv.y & 0x7fffffffu) - tau_hat;
             return ((unsigned long long)(o & lowmask) << 32) | (unsigned long long)(0xffffffffu - cv.x);
         };
-        int top = S + 32;  // bits of the composite still undecided
-        unsigned long long prefix = 0ull;
-        bool take_all = false;
-#pragma unroll 1
-        while (top > 0 && !take_all) {
-            const int width = top < 11 ? top : 11;
-            const int shift = top - width;
-            const int nb = 1 << width;
-            for (int k = threadIdx.x; k < nb; k += kThreads) {
-                local[k] = 0u;
-                merged[k] = 0u;
+        for (uint32_t q0 = 0; q0 < nsurv; q0 += kSelThreads) {  // uniform trip count: the loop holds barriers
+            const uint32_t q = q0 + threadIdx.x;
+            bool kept = false;
+            uint2 cv = make_uint2(0u, 0u);
+            if (q < nsurv) {
+                cv = surv[q];
+                const unsigned long long mine_c = comp_of(cv);
+                uint32_t beaten = 0;
+                for (uint32_t p = 0; p < nsurv; ++p) beaten += (comp_of(surv[p]) > mine_c) ? 1u : 0u;
+                kept = beaten < k_rem;
+                if (beaten == k_rem - 1u) sh_edge[1] = (cv.y & 0x7fffffffu);  // the k-th largest key overall
             }
-            cluster.sync();
-            for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
-                const unsigned long long cm = comp_of(surv[q]);
-                if ((cm >> top) == prefix) atomicAdd(&local[(uint32_t)(cm >> shift) & (uint32_t)(nb - 1)], 1u);
-            }
+            uint32_t tot3;
+            const uint32_t incl = block_inclusive_scan<kSelWarps>(kept ? 1u : 0u, scratch, &tot3);
+            if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
             __syncthreads();
-            for (int k = threadIdx.x; k < nb; k += kThreads) {
-                const uint32_t v = local[k];
-                if (v) atomicAdd(merged0 + k, v);
-            }
-            cluster.sync();
-            {
-                uint32_t tot2;
-                const BinScan sc = scan_from_top(merged0, nb, scratch, &tot2);
-                locate(merged0, nb, sc, k_rem, sh_bin);
-            }
-            __syncthreads();
-            prefix = (prefix << width) | (unsigned long long)sh_bin[0];
-            k_rem -= sh_bin[1];
-            take_all = (sh_bin[2] == k_rem);
-            top = shift;
-            cluster.sync();  // rank 0's histogram has been read by everybody before it is cleared again
-        }
-        // kept survivors: composite >> top >= prefix
-        uint32_t cnt = 0;
-        for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) cnt += ((comp_of(surv[q]) >> top) >= prefix) ? 1u : 0u;
-        uint32_t tot3;
-        const uint32_t incl = block_inclusive_scan(cnt, scratch, &tot3);
-        if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
-        __syncthreads();
-        uint32_t pos = sh_base + incl - cnt;
-        for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
-            const uint2 cv = surv[q];
-            if ((comp_of(cv) >> top) >= prefix) {
+            if (kept) {
+                const uint32_t pos = sh_base + incl - 1u;
                 if (pos < kb) {
                     b.idx[slot0 + pos] = (int32_t)cv.x;
                     b.val[slot0 + pos] = __uint_as_float(cv.y);
                 } else {
                     atomicOr(b.status, 1u);
                 }
-                ++pos;
             }
+            __syncthreads();
         }
-        // decided low key bits of the threshold
-        const unsigned long long lowbits = top >= 32 ? (prefix << (top - 32)) : (prefix >> (32 - top));
-        tau += (uint32_t)lowbits & lowmask;
+        tau = sh_edge[1];
     }
     if (rank == 0 && threadIdx.x == 0) {
         uint32_t edge;
@@ -863,7 +835,7 @@ static cudaError_t launch_select_list(compams_context* c, const int32_t* list, i
     if (nlist == 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((int64_t)c->n * nlist * cluster), 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(kSelThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = c->stream;
     cudaLaunchAttribute attr[1];
