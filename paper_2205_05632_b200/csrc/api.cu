@@ -116,10 +116,16 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
     c->seg_cap_host.clear();
     for (const SegInfo& si : segs) c->seg_cap_host.push_back(si.cap);
     if (topk) {
+        // Short candidate lists get one CTA each, long ones a cluster of CTAs. A cluster finishes one
+        // list sooner, but far fewer clusters than CTAs fit on the GPU at once: with many long lists
+        // (layer-wise selection over many workers) one CTA per list has the higher throughput.
+        size_t n_long = 0;
+        for (const SegInfo& si : segs) n_long += si.cap > (uint32_t)kSelectSingleMax ? 1 : 0;
+        const uint32_t single_max = (n_long * (size_t)c->n >= 64) ? (1u << 20) : (uint32_t)kSelectSingleMax;
         std::vector<int32_t> small_l, big_l;
         for (size_t s = 0; s < segs.size(); ++s) {
             if (segs[s].cap == 0) continue;  // never predicts: always the dense passes, no select needed
-            (segs[s].cap <= (uint32_t)kSelectSingleMax ? small_l : big_l).push_back((int32_t)s);
+            (segs[s].cap <= single_max ? small_l : big_l).push_back((int32_t)s);
         }
         RC(dev_upload(c, &c->sel_small, small_l));
         RC(dev_upload(c, &c->sel_big, big_l));
