@@ -63,13 +63,14 @@ __global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t
     }
 }
 
-__global__ void __launch_bounds__(kThreads) amsgrad_from_acc_kernel(int64_t d, double* __restrict__ acc,
-                                                                    float* __restrict__ gbar, float* __restrict__ m,
-                                                                    float* __restrict__ v, float* __restrict__ vhat,
-                                                                    float* __restrict__ theta, HyperParams hp) {
+// One float4 group per thread.
+__global__ void __launch_bounds__(kThreads, 6) amsgrad_from_acc_kernel(int64_t d, double* __restrict__ acc,
+                                                                       float* __restrict__ gbar, float* __restrict__ m,
+                                                                       float* __restrict__ v, float* __restrict__ vhat,
+                                                                       float* __restrict__ theta, HyperParams hp) {
     const int64_t groups = d >> 2;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < groups; q += stride) {
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < groups) {
         const int64_t j = q << 2;
         double2 a01 = *reinterpret_cast<const double2*>(acc + j);
         double2 a23 = *reinterpret_cast<const double2*>(acc + j + 2);
@@ -105,13 +106,6 @@ __global__ void __launch_bounds__(kThreads) amsgrad_from_acc_kernel(int64_t d, d
     }
 }
 
-static int grid_for(const compams_context* c, int64_t work_items, int ctas_per_sm) {
-    int64_t want = (work_items + kThreads - 1) / kThreads;
-    int64_t cap = (int64_t)c->num_sms * ctas_per_sm;
-    if (want < 1) want = 1;
-    return (int)(want < cap ? want : cap);
-}
-
 cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, float* theta) {
     int64_t groups = c->d >> 2;
     int grid = (int)((groups + kThreads - 1) / kThreads);
@@ -122,7 +116,9 @@ cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, fl
 }
 
 cudaError_t launch_amsgrad(compams_context* c, float* theta) {
-    int grid = grid_for(c, c->d >> 2, 8);
+    int64_t groups = c->d >> 2;
+    int grid = (int)((groups + kThreads - 1) / kThreads);
+    if (grid < 1) grid = 1;
     amsgrad_from_acc_kernel<<<grid, kThreads, 0, c->stream>>>(c->d, c->tk.acc, c->gbar, c->m, c->v, c->vhat, theta,
                                                               c->hp);
     return cudaGetLastError();

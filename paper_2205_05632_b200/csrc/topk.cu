@@ -793,21 +793,17 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 // scatter: acc[j] += x_ij over all kept (i, j); binary64 atomics, exact hence order-independent.
 // The same walk zeroes e at the kept coordinates (they were left holding x by the sweep).
 
-__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(int64_t K, int64_t d, int32_t n,
+__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(int64_t K, int64_t d, int64_t count,
                                                                 const int32_t* __restrict__ idx,
                                                                 const float* __restrict__ val,
                                                                 double* __restrict__ acc, float* __restrict__ E) {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int i = 0; i < n; ++i) {
-        const int32_t* ix = idx + (size_t)i * (size_t)K;
-        const float* vx = val + (size_t)i * (size_t)K;
-        float* e = E + (size_t)i * (size_t)d;
-        for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < K; p += stride) {
-            const int32_t j = ix[p];
-            atomicAdd(acc + j, (double)vx[p]);
-            e[j] = 0.0f;
-        }
-    }
+    // one (index, value) pair per thread: every pair's read-modify-write is in flight at once
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= count) return;
+    const int64_t i = p / K;
+    const int32_t j = __ldg(idx + p);
+    atomicAdd(acc + j, (double)__ldg(val + p));
+    E[(size_t)i * (size_t)d + (size_t)j] = 0.0f;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -889,8 +885,9 @@ cudaError_t launch_topk_ties(compams_context* c) {
 }
 
 cudaError_t launch_topk_scatter(compams_context* c) {
-    const int grid = persistent_grid(c, (c->K + kThreads - 1) / kThreads, 8);
-    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->K, c->d, c->n, c->tk.idx, c->tk.val, c->tk.acc, c->E);
+    const int64_t count = (int64_t)c->n * c->K;
+    const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
+    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->K, c->d, count, c->tk.idx, c->tk.val, c->tk.acc, c->E);
     return cudaGetLastError();
 }
 
