@@ -76,11 +76,10 @@ enum compams_kernel {
     COMPAMS_K_BS_APPLY = 2,           /* Block-Sign: segmented average over workers fused with AMSGrad        */
     COMPAMS_K_BS_MATERIALIZE = 3,     /* Block-Sign: turn the stored x into e when E is read                  */
     COMPAMS_K_TOPK_SWEEP = 4,         /* Top-k: EF add, x written to E, candidates above the predicted threshold */
-    COMPAMS_K_TOPK_HIST = 5,          /* Top-k dense passes: radix histograms over x                          */
-    COMPAMS_K_TOPK_FIND = 6,          /* Top-k dense passes: locate the threshold bin of a pass               */
-    COMPAMS_K_TOPK_COLLECT = 7,       /* Top-k dense passes: emit (index, value), count threshold ties        */
-    COMPAMS_K_TOPK_TIES = 8,          /* Top-k: lowest-index ties at the threshold; closes the step per segment */
-    COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: sparse scatter-accumulate into the averaged gradient          */
+    COMPAMS_K_TOPK_DENSE = 5,         /* Top-k dense passes (one cooperative launch): radix histograms over x,
+                                         threshold search, emission, lowest-index ties                        */
+    /* 6, 7, 8: unused */
+    COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: closes the step per segment; sparse scatter-accumulate         */
     COMPAMS_K_AMSGRAD = 10,           /* Top-k: AMSGrad update from the accumulated average                   */
     COMPAMS_K_TOPK_SMALL = 11,        /* Top-k: whole small blocks selected inside shared memory              */
     COMPAMS_K_TOPK_SELECT = 12,       /* Top-k: exact selection inside the candidate lists                    */

@@ -285,14 +285,7 @@ int step_device(compams_context* c, const float* grads, float* theta) {
     if (c->tab.ntiles > 0) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_SELECT, [&] { return launch_topk_select(c); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 1); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 1); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 2); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 2); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_HIST, [&] { return launch_topk_hist(c, 3); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_FIND, [&] { return launch_topk_find(c, 3); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_COLLECT, [&] { return launch_topk_collect(c); }));
-        RC(run_kernel(c, COMPAMS_K_TOPK_TIES, [&] { return launch_topk_ties(c); }));
+        RC(run_kernel(c, COMPAMS_K_TOPK_DENSE, [&] { return launch_topk_dense(c); }));
     }
     RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c); }));
     RC(run_kernel(c, COMPAMS_K_AMSGRAD, [&] { return launch_amsgrad(c, theta); }));
@@ -488,8 +481,8 @@ const char* compams_error_string(int status) {
 
 const char* compams_kernel_name(int32_t kernel) {
     static const char* names[COMPAMS_K_COUNT] = {
-        "dense_mean_amsgrad", "bs_sweep", "bs_apply", "bs_materialize", "topk_sweep", "topk_hist",
-        "topk_find", "topk_collect", "topk_ties", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
+        "dense_mean_amsgrad", "bs_sweep", "bs_apply", "bs_materialize", "topk_sweep", "topk_dense",
+        "unused", "unused", "unused", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
     return (kernel >= 0 && kernel < COMPAMS_K_COUNT) ? names[kernel] : "unknown";
 }
 

@@ -110,6 +110,7 @@ struct compams_context {
     int32_t* sel_small = nullptr;  // tiled blocks whose candidate lists one CTA selects from
     int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists a cluster selects from
     int n_sel_small = 0, n_sel_big = 0;
+    int dense_grid = 0;  // CTAs of the cooperative dense-pass kernel (0: not yet sized)
     float* scales[2] = {nullptr, nullptr};
     int scales_cur = 0;
     bool e_is_x = false;  // Block-Sign: E holds the corrected gradient x of the last step, not e
@@ -145,10 +146,7 @@ cudaError_t launch_bs_materialize(compams_context* c);
 cudaError_t launch_topk_small(compams_context* c, const float* grads);
 cudaError_t launch_topk_sweep(compams_context* c, const float* grads);
 cudaError_t launch_topk_select(compams_context* c);
-cudaError_t launch_topk_hist(compams_context* c, int pass);
-cudaError_t launch_topk_find(compams_context* c, int pass);
-cudaError_t launch_topk_collect(compams_context* c);
-cudaError_t launch_topk_ties(compams_context* c);
+cudaError_t launch_topk_dense(compams_context* c);
 cudaError_t launch_topk_scatter(compams_context* c);
 cudaError_t launch_amsgrad(compams_context* c, float* theta);
 

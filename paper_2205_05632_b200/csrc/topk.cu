@@ -18,14 +18,15 @@
 //                   emitted, the bin's few candidates go to rank 0's shared memory, which orders them
 //                   by (key, lower index first), keeps the best and predicts the next tau_hat.
 //                   Otherwise the segment is marked for the dense passes.
-//   Dense passes (only for marked segments; exact for any input, e.g. all-equal values):
-//     topk_hist<1..3> / topk_find<1..3>  three histogram passes over x, 11 + 10 + 10 key bits
-//     topk_collect  keys above the threshold are emitted; threshold ties too unless only some fit,
+//   Dense passes (only for marked segments; exact for any input, e.g. all-equal values), one
+//   cooperative kernel topk_dense whose stages are separated by grid-wide barriers:
+//     hist<1..3> / find<1..3>  three histogram passes over x, 11 + 10 + 10 key bits
+//     collect       keys above the threshold are emitted; threshold ties too unless only some fit,
 //                   in which case they are counted per tile
-//     topk_ties     takes the lowest-index threshold ties, tile by tile in index order; also closes
-//                   the step for every segment (count check, counters reset)
-//   topk_scatter    walks the (index, value) messages: sum_i g~_i accumulated into a binary64
-//                   buffer (line 12) and e zeroed at every kept coordinate (line 8: e = x - x)
+//     ties          takes the lowest-index threshold ties, tile by tile in index order
+//   topk_scatter    closes the step per segment (count check, counters reset) and walks the
+//                   (index, value) messages: sum_i g~_i accumulated into a binary64 buffer (line 12),
+//                   e zeroed at every kept coordinate (line 8: e = x - x)
 #include <cooperative_groups.h>
 
 #include "context.h"
@@ -444,10 +445,8 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
 // dense passes, only for segments marked `fallback`
 
 template <int PASS>
-__global__ void __launch_bounds__(kThreads) topk_hist_kernel(Tables t, TopkBuffers b) {
+__device__ __forceinline__ void dense_hist(const Tables& t, const TopkBuffers& b, uint32_t* sh) {
     constexpr int NB = (PASS == 1) ? kBins1 : kBins23;
-    __shared__ uint32_t sh[NB];
-    if (*b.dense_count == 0u) return;  // every segment was decided inside its candidate list
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t total = (int64_t)t.n * t.ntiles;
     for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
@@ -487,11 +486,8 @@ __global__ void __launch_bounds__(kThreads) topk_hist_kernel(Tables t, TopkBuffe
 }
 
 template <int NBINS, int BITS, int PASS>
-__global__ void __launch_bounds__(kThreads) topk_find_kernel(Tables t, TopkBuffers b) {
-    __shared__ uint32_t scratch[kWarps];
+__device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b, size_t sg, uint32_t* scratch) {
     constexpr int PER = NBINS / kThreads;
-    if (*b.dense_count == 0u) return;
-    const size_t sg = blockIdx.x;
     SegState* st = b.seg + sg;
     if (st->fallback == 0u) return;
     const SegInfo* si = t.segs + (sg % (size_t)t.nseg);
@@ -555,10 +551,9 @@ __global__ void __launch_bounds__(kThreads) topk_find_kernel(Tables t, TopkBuffe
     if (threadIdx.x == 0 && total < k_rem) atomicOr(b.status, 2u);
 }
 
-__global__ void __launch_bounds__(kThreads) topk_collect_kernel(Tables t, TopkBuffers b) {
-    __shared__ uint32_t scratch[kWarps];
-    __shared__ uint32_t sh_base;
-    if (*b.dense_count == 0u) return;
+__device__ __forceinline__ void dense_collect(const Tables& t, const TopkBuffers& b, uint32_t* scratch,
+                                              uint32_t* sh_base_p) {
+    uint32_t& sh_base = *sh_base_p;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t total = (int64_t)t.n * t.ntiles;
     for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
@@ -623,32 +618,20 @@ __global__ void __launch_bounds__(kThreads) topk_collect_kernel(Tables t, TopkBu
     }
 }
 
-// Closes the step for one segment: if the dense passes left threshold ties to order, takes those
-// with the lowest index; then checks that exactly k_b entries were emitted and resets the counters.
-__global__ void __launch_bounds__(kThreads) topk_ties_kernel(Tables t, TopkBuffers b) {
-    __shared__ uint32_t scratch[kWarps];
-    __shared__ uint32_t sh_c[kThreads], sh_excl[kThreads];
-    const size_t sg = blockIdx.x;
+// When the dense passes left threshold ties to order, takes those with the lowest index, tile by
+// tile. The ties land in the message slots after the `emit_count` winners; the count itself is
+// checked (with the ties added) when the step is closed.
+__device__ __forceinline__ void dense_ties(const Tables& t, const TopkBuffers& b, size_t sg, uint32_t* scratch,
+                                           uint32_t* sh_c, uint32_t* sh_excl) {
     const int i = (int)(sg / (size_t)t.nseg);
     const SegInfo* si = t.segs + (sg % (size_t)t.nseg);
-    SegState* st = b.seg + sg;
+    const SegState* st = b.seg + sg;
+    if (st->fallback == 0u || st->need_order == 0u) return;
     const uint32_t kb = si->kb;
     const uint32_t emitted = st->emit_count;
-    const bool dense = st->fallback != 0u;
-    const bool need_order = dense && st->need_order != 0u;
     const uint32_t tau = st->tau;
-    const uint32_t want = need_order ? st->ties_take : 0u;
-    __syncthreads();  // every thread has read the state before thread 0 resets it
-    if (threadIdx.x == 0) {
-        if (emitted + want != kb) atomicOr(b.status, 1u);
-        if (dense) atomicAdd(b.status + 1, 1u);              // selections decided by the dense passes
-        if (dense && si->cap) atomicSub(b.dense_count, 1u);  // back to the number of blocks that never predict
-        st->emit_count = 0u;
-        st->cand_count = 0u;
-        st->fallback = si->cap ? 0u : 1u;  // blocks without a candidate buffer always take the dense passes
-        st->need_order = 0u;
-    }
-    if (!need_order || emitted + want != kb) return;
+    const uint32_t want = st->ties_take;
+    if (emitted + want != kb) return;  // inconsistent: reported when the step is closed
     const int tile0 = si->tile0, tile_end = si->tile0 + si->ntile_b;
     const int64_t o = si->o;
     const int len = si->len;
@@ -696,6 +679,47 @@ __global__ void __launch_bounds__(kThreads) topk_ties_kernel(Tables t, TopkBuffe
         __syncthreads();
     }
     if (threadIdx.x == 0 && taken < want) atomicOr(b.status, 1u);
+}
+
+// All dense passes in one cooperative launch: the grid is resident as a whole and the passes are
+// separated by grid-wide barriers. When no segment is marked every CTA returns at once, so in the
+// steady state the dense path costs one empty launch per step.
+__global__ void __launch_bounds__(kThreads) topk_dense_kernel(Tables t, TopkBuffers b) {
+    __shared__ uint32_t sh[kBins1];
+    __shared__ uint32_t scratch[kWarps];
+    __shared__ uint32_t sh_c[kThreads], sh_excl[kThreads];
+    __shared__ uint32_t sh_base;
+    // the same word for every CTA; it only changes when the step is closed, in a later kernel
+    if (*b.dense_count == 0u) return;
+    cg::grid_group grid = cg::this_grid();
+    const size_t nsg = (size_t)t.n * (size_t)t.nseg;
+    dense_hist<1>(t, b, sh);
+    grid.sync();
+    for (size_t sg = blockIdx.x; sg < nsg; sg += gridDim.x) {
+        dense_find<kBins1, 11, 1>(t, b, sg, scratch);
+        __syncthreads();
+    }
+    grid.sync();
+    dense_hist<2>(t, b, sh);
+    grid.sync();
+    for (size_t sg = blockIdx.x; sg < nsg; sg += gridDim.x) {
+        dense_find<kBins23, 10, 2>(t, b, sg, scratch);
+        __syncthreads();
+    }
+    grid.sync();
+    dense_hist<3>(t, b, sh);
+    grid.sync();
+    for (size_t sg = blockIdx.x; sg < nsg; sg += gridDim.x) {
+        dense_find<kBins23, 10, 3>(t, b, sg, scratch);
+        __syncthreads();
+    }
+    grid.sync();
+    dense_collect(t, b, scratch, &sh_base);
+    grid.sync();
+    for (size_t sg = blockIdx.x; sg < nsg; sg += gridDim.x) {
+        dense_ties(t, b, sg, scratch, sh_c, sh_excl);
+        __syncthreads();
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -793,17 +817,29 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 // scatter: acc[j] += x_ij over all kept (i, j); binary64 atomics, exact hence order-independent.
 // The same walk zeroes e at the kept coordinates (they were left holding x by the sweep).
 
-__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(int64_t K, int64_t d, int64_t count,
-                                                                const int32_t* __restrict__ idx,
-                                                                const float* __restrict__ val,
-                                                                double* __restrict__ acc, float* __restrict__ E) {
-    // one (index, value) pair per thread: every pair's read-modify-write is in flight at once
+__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count) {
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // the first n * nseg threads also close the step for one large-block segment each: exactly k_b
+    // entries must have been emitted; counters go back to their resting values
+    if (p < (int64_t)t.n * t.nseg) {
+        const SegInfo* si = t.segs + (p % t.nseg);
+        SegState* st = b.seg + p;
+        const bool dense = st->fallback != 0u;
+        const uint32_t ties = (dense && st->need_order) ? st->ties_take : 0u;
+        if (st->emit_count + ties != si->kb) atomicOr(b.status, 1u);
+        if (dense) atomicAdd(b.status + 1, 1u);              // selections decided by the dense passes
+        if (dense && si->cap) atomicSub(b.dense_count, 1u);  // back to the number of blocks that never predict
+        st->emit_count = 0u;
+        st->cand_count = 0u;
+        st->fallback = si->cap ? 0u : 1u;  // blocks without a candidate buffer always take the dense passes
+        st->need_order = 0u;
+    }
+    // one (index, value) pair per thread: every pair's read-modify-write is in flight at once
     if (p >= count) return;
-    const int64_t i = p / K;
-    const int32_t j = __ldg(idx + p);
-    atomicAdd(acc + j, (double)__ldg(val + p));
-    E[(size_t)i * (size_t)d + (size_t)j] = 0.0f;
+    const int64_t i = p / b.K;
+    const int32_t j = __ldg(b.idx + p);
+    atomicAdd(b.acc + j, (double)__ldg(b.val + p));
+    b.E[(size_t)i * (size_t)t.d + (size_t)j] = 0.0f;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -850,44 +886,23 @@ cudaError_t launch_topk_select(compams_context* c) {
     return launch_select_list(c, c->sel_big, c->n_sel_big, kSelectCluster);
 }
 
-cudaError_t launch_topk_find(compams_context* c, int pass) {
-    const unsigned grid = (unsigned)((int64_t)c->n * c->tab.nseg);
-    if (pass == 1)
-        topk_find_kernel<kBins1, 11, 1><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    else if (pass == 2)
-        topk_find_kernel<kBins23, 10, 2><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    else
-        topk_find_kernel<kBins23, 10, 3><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_topk_hist(compams_context* c, int pass) {
-    const int grid = persistent_grid(c, (int64_t)c->n * c->tab.ntiles, 8);
-    if (pass == 1)
-        topk_hist_kernel<1><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    else if (pass == 2)
-        topk_hist_kernel<2><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    else
-        topk_hist_kernel<3><<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_topk_collect(compams_context* c) {
-    const int grid = persistent_grid(c, (int64_t)c->n * c->tab.ntiles, 6);
-    topk_collect_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_topk_ties(compams_context* c) {
-    const unsigned grid = (unsigned)((int64_t)c->n * c->tab.nseg);
-    topk_ties_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
-    return cudaGetLastError();
+cudaError_t launch_topk_dense(compams_context* c) {
+    if (c->dense_grid == 0) {
+        int per_sm = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_dense_kernel, kThreads, 0);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+        c->dense_grid = per_sm * c->num_sms;  // every CTA resident at once, as a cooperative launch requires
+    }
+    void* args[] = {(void*)&c->tab, (void*)&c->tk};
+    return cudaLaunchCooperativeKernel((const void*)topk_dense_kernel, dim3((unsigned)c->dense_grid), dim3(kThreads), args,
+                                       0, c->stream);
 }
 
 cudaError_t launch_topk_scatter(compams_context* c) {
-    const int64_t count = (int64_t)c->n * c->K;
+    const int64_t count = (int64_t)c->n * c->K;  // >= n * nseg: every block keeps at least one entry
     const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
-    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->K, c->d, count, c->tk.idx, c->tk.val, c->tk.acc, c->E);
+    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count);
     return cudaGetLastError();
 }
 
