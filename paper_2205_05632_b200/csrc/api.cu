@@ -202,6 +202,18 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &t.tile_ties, (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &t.cand, (size_t)n * (size_t)t.cand_total, false));
         RC(dev_alloc(c, &t.acc, (size_t)d));
+        {
+            // kept entries are handed to the server grouped by coordinate range: room for four times the
+            // average load of a bucket, the rare excess goes through the binary64 accumulator
+            t.nbucket = (int32_t)((d + kBucketSpan - 1) / kBucketSpan);
+            const int64_t avg = ((int64_t)n * c->K + t.nbucket - 1) / t.nbucket;
+            int64_t cap = 4 * avg + 64;
+            if (cap > (int64_t)n * kBucketSpan) cap = (int64_t)n * kBucketSpan;
+            t.bucket_cap = (int32_t)((cap + 31) / 32 * 32);
+            RC(dev_alloc(c, &t.bucket, (size_t)t.nbucket * (size_t)t.bucket_cap, false));
+            RC(dev_alloc(c, &t.bcount, (size_t)t.nbucket));
+            RC(dev_alloc(c, &t.bdirty, (size_t)t.nbucket));
+        }
         t.status = c->status;
         t.gbar = c->gbar;
         t.m = c->m;

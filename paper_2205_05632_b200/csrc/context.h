@@ -14,6 +14,7 @@ namespace compams {
 constexpr int kSmallMax = 4096;    // Top-k blocks up to this size are selected inside one CTA's shared memory
 constexpr int kBins1 = 2048;       // radix pass 1: key bits 30..20
 constexpr int kBins23 = 1024;      // radix passes 2, 3: key bits 19..10, 9..0
+constexpr int kBucketSpan = 1024;  // coordinates per server bucket: one CTA of the Top-k AMSGrad kernel
 constexpr int kMaxTimed = 4096;    // event pairs kept for per-kernel timing
 
 constexpr uint32_t kNoPrediction = 0xffffffffu;  // tau_hat value that no key reaches
@@ -79,7 +80,12 @@ struct TopkBuffers {
     uint2* cand;               // [n, cand_total] (coordinate, bits of x) pairs collected by the sweep
     int64_t cand_total;        // candidate slots per worker
     uint32_t* dense_count;     // [1] segments currently marked for the dense passes
-    double* acc;               // [d] binary64 accumulator of the worker average
+    double* acc;               // [d] binary64 accumulator, used only by entries that overflow their bucket
+    uint2* bucket;             // [nbucket, bucket_cap] (coordinate inside the bucket, bits of x) per kept entry
+    uint32_t* bcount;          // [nbucket] entries appended this step (may exceed bucket_cap)
+    uint32_t* bdirty;          // [nbucket] 1: some entries of this bucket went to acc instead
+    int32_t bucket_cap;
+    int32_t nbucket;
     uint32_t* status;
     float *gbar, *m, *v, *vhat;
 };

@@ -4,9 +4,9 @@
 // so e stays 0), fused with the AMSGrad update (lines 13-16). One pass over G [n, d] and the
 // four state vectors: (4n + 32) bytes per coordinate plus 4 for gbar.
 //
-// amsgrad_from_acc: the server update of the Top-k path. The scatter kernel has accumulated
-// sum_i g~_i in a binary64 buffer; this kernel rounds it, divides by n, clears the buffer for
-// the next step and applies lines 13-16.
+// amsgrad_bucket: the server update of the Top-k path. The scatter kernel has grouped the kept
+// (coordinate, value) entries of all workers by coordinate range; one CTA per range sums them in
+// binary64 in shared memory, rounds, divides by n and applies lines 13-16.
 #include "context.h"
 
 namespace compams {
@@ -63,46 +63,82 @@ __global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t
     }
 }
 
-// One float4 group per thread.
-__global__ void __launch_bounds__(kThreads, 6) amsgrad_from_acc_kernel(int64_t d, double* __restrict__ acc,
-                                                                       float* __restrict__ gbar, float* __restrict__ m,
-                                                                       float* __restrict__ v, float* __restrict__ vhat,
-                                                                       float* __restrict__ theta, HyperParams hp) {
-    const int64_t groups = d >> 2;
-    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (q < groups) {
-        const int64_t j = q << 2;
-        double2 a01 = *reinterpret_cast<const double2*>(acc + j);
-        double2 a23 = *reinterpret_cast<const double2*>(acc + j + 2);
-        float4 mm = *reinterpret_cast<const float4*>(m + j);
-        float4 vv = *reinterpret_cast<const float4*>(v + j);
-        float4 vh = *reinterpret_cast<const float4*>(vhat + j);
-        float4 th = *reinterpret_cast<const float4*>(theta + j);
-        float4 gb = make_float4(mean_from_acc(a01.x, hp.nf), mean_from_acc(a01.y, hp.nf), mean_from_acc(a23.x, hp.nf),
-                                mean_from_acc(a23.y, hp.nf));
+// Server update of the Top-k path, one CTA per bucket of kBucketSpan coordinates: the bucket's kept
+// entries (all workers) are summed in binary64 in shared memory - exact, hence independent of the
+// order - then gbar = (float)sum / n and Algorithm 2, lines 13-16. Entries that did not fit their
+// bucket were added to acc[] by the scatter kernel and are folded in (and acc cleared) here.
+__global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, TopkBuffers b, float* __restrict__ theta,
+                                                                     HyperParams hp) {
+    static_assert(kBucketSpan == 4 * kThreads, "one float4 group per thread");
+    __shared__ double sacc[kBucketSpan];
+    const uint32_t T = blockIdx.x;
+    const int loc = (int)threadIdx.x * 4;
+    const int64_t j = (int64_t)T * kBucketSpan + loc;
+    const bool full = j + 3 < d;
+    // the state of this thread's four coordinates is requested first, so that it is in flight
+    // while the bucket's entries are summed
+    float4 mm = make_float4(0.f, 0.f, 0.f, 0.f), vv = mm, vh = mm, th = mm;
+    if (full) {
+        mm = *reinterpret_cast<const float4*>(b.m + j);
+        vv = *reinterpret_cast<const float4*>(b.v + j);
+        vh = *reinterpret_cast<const float4*>(b.vhat + j);
+        th = *reinterpret_cast<const float4*>(theta + j);
+    }
+    const uint32_t appended = b.bcount[T];
+    const uint32_t cnt = appended < (uint32_t)b.bucket_cap ? appended : (uint32_t)b.bucket_cap;
+    const bool dirty = b.bdirty[T] != 0u;
+    sacc[loc] = 0.0;
+    sacc[loc + 1] = 0.0;
+    sacc[loc + 2] = 0.0;
+    sacc[loc + 3] = 0.0;
+    __syncthreads();
+    const uint2* ent = b.bucket + (size_t)T * (size_t)b.bucket_cap;
+    for (uint32_t e = threadIdx.x; e < cnt; e += kThreads) {
+        const uint2 cv = ent[e];
+        atomicAdd(&sacc[cv.x], (double)__uint_as_float(cv.y));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        b.bcount[T] = 0u;
+        b.bdirty[T] = 0u;
+    }
+    if (j >= d) return;
+    double a[4] = {sacc[loc], sacc[loc + 1], sacc[loc + 2], sacc[loc + 3]};
+    if (full) {
+        if (dirty) {
+            const double2 x01 = *reinterpret_cast<const double2*>(b.acc + j);
+            const double2 x23 = *reinterpret_cast<const double2*>(b.acc + j + 2);
+            a[0] += x01.x; a[1] += x01.y; a[2] += x23.x; a[3] += x23.y;
+            *reinterpret_cast<double2*>(b.acc + j) = make_double2(0.0, 0.0);
+            *reinterpret_cast<double2*>(b.acc + j + 2) = make_double2(0.0, 0.0);
+        }
+        float4 gb = make_float4(mean_from_acc(a[0], hp.nf), mean_from_acc(a[1], hp.nf), mean_from_acc(a[2], hp.nf),
+                                mean_from_acc(a[3], hp.nf));
         amsgrad_update(gb.x, mm.x, vv.x, vh.x, th.x, hp);
         amsgrad_update(gb.y, mm.y, vv.y, vh.y, th.y, hp);
         amsgrad_update(gb.z, mm.z, vv.z, vh.z, th.z, hp);
         amsgrad_update(gb.w, mm.w, vv.w, vh.w, th.w, hp);
-        *reinterpret_cast<double2*>(acc + j) = make_double2(0.0, 0.0);
-        *reinterpret_cast<double2*>(acc + j + 2) = make_double2(0.0, 0.0);
-        *reinterpret_cast<float4*>(gbar + j) = gb;
-        *reinterpret_cast<float4*>(m + j) = mm;
-        *reinterpret_cast<float4*>(v + j) = vv;
-        *reinterpret_cast<float4*>(vhat + j) = vh;
+        *reinterpret_cast<float4*>(b.gbar + j) = gb;
+        *reinterpret_cast<float4*>(b.m + j) = mm;
+        *reinterpret_cast<float4*>(b.v + j) = vv;
+        *reinterpret_cast<float4*>(b.vhat + j) = vh;
         *reinterpret_cast<float4*>(theta + j) = th;
-    }
-    if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
-        const int64_t j = (groups << 2) + threadIdx.x;
-        float gb = mean_from_acc(acc[j], hp.nf);
-        acc[j] = 0.0;
-        float mm = m[j], vv = v[j], vh = vhat[j], th = theta[j];
-        amsgrad_update(gb, mm, vv, vh, th, hp);
-        gbar[j] = gb;
-        m[j] = mm;
-        v[j] = vv;
-        vhat[j] = vh;
-        theta[j] = th;
+    } else {
+        for (int k = 0; k < 4 && j + k < d; ++k) {
+            double ak = a[k];
+            if (dirty) {
+                ak += b.acc[j + k];
+                b.acc[j + k] = 0.0;
+            }
+            const float gb = mean_from_acc(ak, hp.nf);
+            float m1 = b.m[j + k], v1 = b.v[j + k], h1 = b.vhat[j + k], t1 = theta[j + k];
+            amsgrad_update(gb, m1, v1, h1, t1, hp);
+            b.gbar[j + k] = gb;
+            b.m[j + k] = m1;
+            b.v[j + k] = v1;
+            b.vhat[j + k] = h1;
+            theta[j + k] = t1;
+        }
     }
 }
 
@@ -116,11 +152,7 @@ cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, fl
 }
 
 cudaError_t launch_amsgrad(compams_context* c, float* theta) {
-    int64_t groups = c->d >> 2;
-    int grid = (int)((groups + kThreads - 1) / kThreads);
-    if (grid < 1) grid = 1;
-    amsgrad_from_acc_kernel<<<grid, kThreads, 0, c->stream>>>(c->d, c->tk.acc, c->gbar, c->m, c->v, c->vhat, theta,
-                                                              c->hp);
+    amsgrad_bucket_kernel<<<(unsigned)c->tk.nbucket, kThreads, 0, c->stream>>>(c->d, c->tk, theta, c->hp);
     return cudaGetLastError();
 }
 

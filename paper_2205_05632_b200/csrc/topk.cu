@@ -25,8 +25,8 @@
 //                   in which case they are counted per tile
 //     ties          takes the lowest-index threshold ties, tile by tile in index order
 //   topk_scatter    closes the step per segment (count check, counters reset) and walks the
-//                   (index, value) messages: sum_i g~_i accumulated into a binary64 buffer (line 12),
-//                   e zeroed at every kept coordinate (line 8: e = x - x)
+//                   (index, value) messages: each pair is appended to the bucket of its coordinate range
+//                   for the server kernel (line 12), e zeroed at every kept coordinate (line 8: e = x - x)
 #include <cooperative_groups.h>
 
 #include "context.h"
@@ -834,11 +834,31 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
         st->fallback = si->cap ? 0u : 1u;  // blocks without a candidate buffer always take the dense passes
         st->need_order = 0u;
     }
-    // one (index, value) pair per thread: every pair's read-modify-write is in flight at once
-    if (p >= count) return;
+    // one (index, value) pair per thread. The pair joins the bucket of its coordinate range (slots
+    // handed out with one atomic per warp and bucket); e is zeroed at the kept coordinate.
+    const bool valid = p < count;
+    int32_t j = 0;
+    uint32_t xbits = 0, T = 0xffffffffu;
+    if (valid) {
+        j = __ldg(b.idx + p);
+        xbits = __float_as_uint(__ldg(b.val + p));
+        T = (uint32_t)j / (uint32_t)kBucketSpan;
+    }
+    const int lane = threadIdx.x & 31;
+    const unsigned peers = __match_any_sync(0xffffffffu, T);
+    uint32_t base = 0;
+    const int leader = __ffs(peers) - 1;
+    if (valid && lane == leader) base = atomicAdd(b.bcount + T, (uint32_t)__popc(peers));
+    base = __shfl_sync(0xffffffffu, base, leader);
+    if (!valid) return;
+    const uint32_t pos = base + (uint32_t)__popc(peers & ((1u << lane) - 1u));
+    if (pos < (uint32_t)b.bucket_cap) {
+        b.bucket[(size_t)T * (size_t)b.bucket_cap + pos] = make_uint2((uint32_t)j % (uint32_t)kBucketSpan, xbits);
+    } else {  // a coordinate range kept by far more entries than average: binary64 atomics instead
+        atomicAdd(b.acc + j, (double)__uint_as_float(xbits));
+        b.bdirty[T] = 1u;
+    }
     const int64_t i = p / b.K;
-    const int32_t j = __ldg(b.idx + p);
-    atomicAdd(b.acc + j, (double)__ldg(b.val + p));
     b.E[(size_t)i * (size_t)t.d + (size_t)j] = 0.0f;
 }
 
