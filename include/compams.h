@@ -78,7 +78,8 @@ enum compams_kernel {
     COMPAMS_K_TOPK_SWEEP = 4,         /* Top-k: EF add, x written to E, candidates above the predicted threshold */
     COMPAMS_K_TOPK_DENSE = 5,         /* Top-k dense passes (one cooperative launch): radix histograms over x,
                                          threshold search, emission, lowest-index ties                        */
-    /* 6, 7, 8: unused */
+    COMPAMS_K_TOPK_MATERIALIZE = 6,   /* Top-k: zero e at the coordinates kept in the last step when E is read   */
+    /* 7, 8: unused */
     COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: closes the step per segment; sparse scatter-accumulate         */
     COMPAMS_K_AMSGRAD = 10,           /* Top-k: AMSGrad update from the accumulated average                   */
     COMPAMS_K_TOPK_SMALL = 11,        /* Top-k: whole small blocks selected inside shared memory              */
@@ -166,10 +167,11 @@ int compams_set_lr(compams_handle h, float lr);
  *             compressor, in which case *dev_ptr is null).
  *
  * The contents are those of the last enqueued step once the stream has reached that point;
- * they stay valid until the next compams_step / compams_destroy. Asking for BUF_E of a
- * Block-Sign handle enqueues one extra kernel that turns the stored corrected gradient x into
- * the residual e = x - g~ in place (the step itself defers that subtraction to the next
- * iteration's sweep; values are identical either way).
+ * they stay valid until the next compams_step / compams_destroy. Asking for BUF_E enqueues
+ * one extra kernel that finishes line 8 of Algorithm 2 in place: the step itself leaves the
+ * corrected gradient x in E (Block-Sign: all of it; Top-k: at the kept coordinates, which are
+ * recorded in a bit map) and applies e = x - g~ when E is next read, by the next iteration's sweep
+ * or by this call; the values are identical either way.
  *
  * SIGN_BITS layout: row i has W words; block b starts at word SIGN_WORD_OFFSETS[b]; bit (r % 32)
  * of word SIGN_WORD_OFFSETS[b] + r / 32 is the sign bit of x at coordinate block_offsets[b] + r;

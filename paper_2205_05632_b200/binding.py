@@ -32,7 +32,7 @@ _TYPESTR = {torch.float32: "<f4", torch.int32: "<i4", torch.int64: "<i8"}
 
 KERNELS = {
     "dense_mean_amsgrad": 0, "bs_sweep": 1, "bs_apply": 2, "bs_materialize": 3, "topk_sweep": 4, "topk_dense": 5,
-    "topk_scatter": 9, "amsgrad": 10, "topk_small": 11,
+    "topk_materialize": 6, "topk_scatter": 9, "amsgrad": 10, "topk_small": 11,
     "topk_select": 12, "bs_scales": 13,
 }
 

@@ -202,6 +202,9 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &t.tile_ties, (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &t.cand, (size_t)n * (size_t)t.cand_total, false));
         RC(dev_alloc(c, &t.acc, (size_t)d));
+        t.map_words = (d + 31) / 32;
+        RC(dev_alloc(c, &c->keptmap[0], (size_t)n * (size_t)t.map_words));
+        RC(dev_alloc(c, &c->keptmap[1], (size_t)n * (size_t)t.map_words));
         {
             // kept entries are handed to the server grouped by coordinate range: room for four times the
             // average load of a bucket, the rare excess goes through the binary64 accumulator
@@ -293,6 +296,12 @@ int step_device(compams_context* c, const float* grads, float* theta) {
         RC(run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); }));
         return COMPAMS_OK;
     }
+    // kept coordinates are recorded in a bit map; their e is zeroed when E is next read (by the next
+    // sweep, or by topk_materialize when the caller asks for E)
+    c->map_cur ^= 1;
+    c->tk.kept_cur = c->keptmap[c->map_cur];
+    c->tk.kept_prev = c->e_mask_pending ? c->keptmap[c->map_cur ^ 1] : nullptr;
+    CU(cudaMemsetAsync(c->tk.kept_cur, 0, (size_t)c->n * (size_t)c->tk.map_words * sizeof(uint32_t), c->stream));
     if (c->tk.nsmall > 0) RC(run_kernel(c, COMPAMS_K_TOPK_SMALL, [&] { return launch_topk_small(c, grads); }));
     if (c->tab.ntiles > 0) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
@@ -300,6 +309,7 @@ int step_device(compams_context* c, const float* grads, float* theta) {
         RC(run_kernel(c, COMPAMS_K_TOPK_DENSE, [&] { return launch_topk_dense(c); }));
     }
     RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c); }));
+    c->e_mask_pending = true;
     RC(run_kernel(c, COMPAMS_K_AMSGRAD, [&] { return launch_amsgrad(c, theta); }));
     return COMPAMS_OK;
 }
@@ -418,6 +428,10 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
     const bool sign = c->compressor == COMPAMS_BLOCKSIGN;
     switch (which) {
         case COMPAMS_BUF_E:
+            if (topk && c->e_mask_pending) {
+                RC(run_kernel(c, COMPAMS_K_TOPK_MATERIALIZE, [&] { return launch_topk_materialize(c); }));
+                c->e_mask_pending = false;
+            }
             if (sign && c->e_is_x) {
                 RC(run_kernel(c, COMPAMS_K_BS_MATERIALIZE, [&] { return launch_bs_materialize(c); }));
                 c->e_is_x = false;
@@ -494,7 +508,7 @@ const char* compams_error_string(int status) {
 const char* compams_kernel_name(int32_t kernel) {
     static const char* names[COMPAMS_K_COUNT] = {
         "dense_mean_amsgrad", "bs_sweep", "bs_apply", "bs_materialize", "topk_sweep", "topk_dense",
-        "unused", "unused", "unused", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
+        "topk_materialize", "unused", "unused", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
     return (kernel >= 0 && kernel < COMPAMS_K_COUNT) ? names[kernel] : "unknown";
 }
 

@@ -81,6 +81,10 @@ struct TopkBuffers {
     int64_t cand_total;        // candidate slots per worker
     uint32_t* dense_count;     // [1] segments currently marked for the dense passes
     double* acc;               // [d] binary64 accumulator, used only by entries that overflow their bucket
+    const uint32_t* kept_prev; // [n, map_words] bit j of row i: coordinate j was kept last step and its e is still
+                               // to be zeroed (null when E is up to date)
+    uint32_t* kept_cur;        // [n, map_words] receives this step's kept coordinates
+    int64_t map_words;         // 32-bit words per worker row of a kept map: ceil(d / 32)
     uint2* bucket;             // [nbucket, bucket_cap] (coordinate inside the bucket, bits of x) per kept entry
     uint32_t* bcount;          // [nbucket] entries appended this step (may exceed bucket_cap)
     uint32_t* bdirty;          // [nbucket] 1: some entries of this bucket went to acc instead
@@ -116,6 +120,9 @@ struct compams_context {
     int32_t* sel_small = nullptr;  // tiled blocks whose candidate lists one CTA selects from
     int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists a cluster selects from
     int n_sel_small = 0, n_sel_big = 0;
+    uint32_t* keptmap[2] = {nullptr, nullptr};  // Top-k: kept maps of this and the previous step
+    int map_cur = 0;
+    bool e_mask_pending = false;  // Top-k: E still holds x at the coordinates kept in the last step
     int dense_grid = 0;  // CTAs of the cooperative dense-pass kernel (0: not yet sized)
     float* scales[2] = {nullptr, nullptr};
     int scales_cur = 0;
@@ -153,6 +160,7 @@ cudaError_t launch_topk_small(compams_context* c, const float* grads);
 cudaError_t launch_topk_sweep(compams_context* c, const float* grads);
 cudaError_t launch_topk_select(compams_context* c);
 cudaError_t launch_topk_dense(compams_context* c);
+cudaError_t launch_topk_materialize(compams_context* c);
 cudaError_t launch_topk_scatter(compams_context* c);
 cudaError_t launch_amsgrad(compams_context* c, float* theta);
 

@@ -26,7 +26,8 @@
 //     ties          takes the lowest-index threshold ties, tile by tile in index order
 //   topk_scatter    closes the step per segment (count check, counters reset) and walks the
 //                   (index, value) messages: each pair is appended to the bucket of its coordinate range
-//                   for the server kernel (line 12), e zeroed at every kept coordinate (line 8: e = x - x)
+//                   for the server kernel (line 12) and marked in the kept map: its e is 0 (line 8:
+//                   e = x - x), applied when E is next read (next sweep, or topk_materialize)
 #include <cooperative_groups.h>
 
 #include "context.h"
@@ -71,15 +72,32 @@ __device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int len
 // ------------------------------------------------------------------------------------------
 // sweep: x = g + e -> E; keys >= tau_hat go to the candidate list
 
+// Bits j .. j+3 of one worker's kept map (bit j of the row = coordinate j), in the low 4 bits.
+__device__ __forceinline__ uint32_t kept_bits4(const uint32_t* __restrict__ row, int64_t map_words, uint32_t j) {
+    const uint32_t w = j >> 5, sh = j & 31u;
+    uint32_t bits = __ldg(row + w) >> sh;
+    if (sh > 28u && (int64_t)w + 1 < map_words) bits |= __ldg(row + w + 1) << (32u - sh);
+    return bits & 0xfu;
+}
+
 template <bool FULL>
 __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int r0,
                                                 int warp, int lane, uint32_t tau_hat, uint32_t coord0,
                                                 uint2* sh_cand, uint32_t* sh_cnt, uint32_t* g_cnt, uint2* g_out,
-                                                uint32_t cap) {
+                                                uint32_t cap, const uint32_t* __restrict__ kept, int64_t map_words) {
     const int cg_ = align_class(g), ce = align_class(e);
+    // kept map of this warp's 1024 coordinates: when the block starts on a word boundary, lane l
+    // fetches word l once and the iterations pick their nibbles with shuffles
+    const bool map_fast = kept != nullptr && (coord0 & 31u) == 0u;
+    uint32_t mapw = 0u;
+    if (map_fast) {
+        const int64_t w = (int64_t)((coord0 + (uint32_t)lane_r(r0, warp, 0, 0)) >> 5) + lane;
+        mapw = w < map_words ? __ldg(kept + w) : 0u;
+    }
 #pragma unroll
     for (int bt = 0; bt < kIters / 2; ++bt) {
         float4 gv[2], ev[2];
+        uint32_t kb4[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int r = lane_r(r0, warp, bt * 2 + u, lane);
@@ -96,14 +114,19 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
                 ev[u] = make_float4(et[0], et[1], et[2], et[3]);
             }
+            // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, line 8)
+            kb4[u] = (kept && !map_fast) ? kept_bits4(kept, map_words, coord0 + (uint32_t)r) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int r = lane_r(r0, warp, bt * 2 + u, lane);
+            if (map_fast)  // after the batch's loads have been issued: the shuffle waits for the map word
+                kb4[u] = (__shfl_sync(0xffffffffu, mapw, (bt * 2 + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
             float xs[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                xs[k] = __fadd_rn(lane_elem(gv[u], k), lane_elem(ev[u], k));  // line 7: x = g + e
+                const float ek = ((kb4[u] >> k) & 1u) ? 0.0f : lane_elem(ev[u], k);
+                xs[k] = __fadd_rn(lane_elem(gv[u], k), ek);  // line 7: x = g + e
                 if ((FULL || r + k < len) && mag_key(xs[k]) >= tau_hat) {
                     const uint2 cv = make_uint2(coord0 + (uint32_t)(r + k), __float_as_uint(xs[k]));
                     const uint32_t slot = atomicAdd(sh_cnt, 1u);
@@ -142,12 +165,13 @@ __global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkB
     __syncthreads();
     const float* g = G + (size_t)i * (size_t)t.d + (size_t)ti.o;
     float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
+    const uint32_t* kept = b.kept_prev ? b.kept_prev + (size_t)i * (size_t)b.map_words : nullptr;
     if (ti.r0 + kTile <= ti.len)
         topk_sweep_tile<true>(g, e, ti.len, ti.r0, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
-                              &st->cand_count, out, cap);
+                              &st->cand_count, out, cap, kept, b.map_words);
     else
         topk_sweep_tile<false>(g, e, ti.len, ti.r0, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
-                               &st->cand_count, out, cap);
+                               &st->cand_count, out, cap, kept, b.map_words);
     __syncthreads();
     const uint32_t cnt = sh_cnt;
     if (cnt == 0u) return;
@@ -858,8 +882,25 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
         atomicAdd(b.acc + j, (double)__uint_as_float(xbits));
         b.bdirty[T] = 1u;
     }
+    // the coordinate's e becomes 0 (line 8: e = x - x): recorded in the kept map, applied when E is next read
     const int64_t i = p / b.K;
-    b.E[(size_t)i * (size_t)t.d + (size_t)j] = 0.0f;
+    atomicOr(b.kept_cur + (size_t)i * (size_t)b.map_words + ((uint32_t)j >> 5), 1u << ((uint32_t)j & 31u));
+}
+
+// E holds x at the coordinates kept in the last step: zero them (Algorithm 2, line 8), one thread per word.
+__global__ void __launch_bounds__(kThreads) topk_materialize_kernel(int32_t n, int64_t d, int64_t map_words,
+                                                                    const uint32_t* __restrict__ kept,
+                                                                    float* __restrict__ E) {
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= (int64_t)n * map_words) return;
+    uint32_t w = kept[q];
+    const int64_t i = q / map_words;
+    float* e = E + (size_t)i * (size_t)d + (size_t)(q % map_words) * 32;
+    while (w) {
+        const int k = __ffs(w) - 1;
+        w &= w - 1;
+        e[k] = 0.0f;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -917,6 +958,13 @@ cudaError_t launch_topk_dense(compams_context* c) {
     void* args[] = {(void*)&c->tab, (void*)&c->tk};
     return cudaLaunchCooperativeKernel((const void*)topk_dense_kernel, dim3((unsigned)c->dense_grid), dim3(kThreads), args,
                                        0, c->stream);
+}
+
+cudaError_t launch_topk_materialize(compams_context* c) {
+    const int64_t words = (int64_t)c->n * c->tk.map_words;
+    topk_materialize_kernel<<<(unsigned)((words + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
+        c->n, c->d, c->tk.map_words, c->keptmap[c->map_cur], c->E);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_topk_scatter(compams_context* c) {
