@@ -112,6 +112,17 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
     c->tab.tiles = d_tiles;
     c->tab.nseg = (int32_t)blocks.size();
     c->tab.segs = d_segs;
+    c->segp = SegParams{};
+    if (segs.size() <= (size_t)kParamSegs) {
+        c->segp.nseg = (int32_t)segs.size();
+        for (size_t s = 0; s < segs.size(); ++s) {
+            c->segp.tile0[s] = segs[s].tile0;
+            c->segp.len[s] = segs[s].len;
+            c->segp.blk[s] = segs[s].blk;
+            c->segp.o[s] = segs[s].o;
+        }
+        c->segp.tile0[segs.size()] = (int32_t)tiles.size();
+    }
     c->tk.cand_total = cand_total;
     c->seg_cap_host.clear();
     for (const SegInfo& si : segs) c->seg_cap_host.push_back(si.cap);

@@ -91,11 +91,11 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
 }
 
 __global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffers b, const float* __restrict__ G,
-                                                               int deferred) {
+                                                               int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     const int tile = blockIdx.x;
     const int i = blockIdx.y;
-    const TileInfo ti = load_tile(t.tiles, tile);
+    const TileInfo ti = sp_.nseg ? find_tile(sp_, tile) : load_tile(t.tiles, tile);
     const int blk = ti.blk;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float* g = G + (size_t)i * (size_t)t.d + (size_t)ti.o;
@@ -228,7 +228,7 @@ cudaError_t launch_bs_sweep(compams_context* c, const float* grads) {
     BsBuffers b = c->bs;
     b.scales_prev = c->scales[c->scales_cur ^ 1];
     b.scales_cur = c->scales[c->scales_cur];
-    bs_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, grads, c->e_is_x ? 1 : 0);
+    bs_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, grads, c->e_is_x ? 1 : 0, c->segp);
     return cudaGetLastError();
 }
 

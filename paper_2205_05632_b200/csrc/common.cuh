@@ -36,6 +36,18 @@ struct __align__(16) SegInfo {
     uint32_t cap;      // candidate capacity (0: this block never uses the candidate path)
 };
 
+// The tiled blocks again, small enough to travel as a kernel argument: a CTA of a sweep finds its
+// tile's block in the constant bank instead of waiting for a global-memory table before it can
+// issue its first data load. nseg = 0 when there are too many blocks (the tile table is used).
+constexpr int kParamSegs = 168;
+struct SegParams {
+    int32_t nseg;
+    int32_t tile0[kParamSegs + 1];  // first tile of each tiled block, then the total
+    int32_t len[kParamSegs];
+    int32_t blk[kParamSegs];
+    int64_t o[kParamSegs];
+};
+
 // AMSGrad hyper-parameters as the fp32 numbers every kernel uses (Algorithm 1).
 struct HyperParams {
     float lr, beta1, beta2, omb1, omb2, eps, nf;  // omb = 1 - beta (fp32), nf = (float)n
@@ -124,6 +136,24 @@ __device__ __forceinline__ TileInfo load_tile(const TileInfo* tiles, int tile) {
     ti.seg = b.y;
     ti.tile0 = b.z;
     ti.ntile_b = b.w;
+    return ti;
+}
+
+// The same record from the kernel-argument copy of the block list (binary search over tile0).
+__device__ __forceinline__ TileInfo find_tile(const SegParams& sp, int tile) {
+    int lo = 0, hi = sp.nseg - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (sp.tile0[mid] <= tile) lo = mid; else hi = mid - 1;
+    }
+    TileInfo ti;
+    ti.o = sp.o[lo];
+    ti.len = sp.len[lo];
+    ti.r0 = (tile - sp.tile0[lo]) * kTile;
+    ti.blk = sp.blk[lo];
+    ti.seg = lo;
+    ti.tile0 = sp.tile0[lo];
+    ti.ntile_b = sp.tile0[lo + 1] - sp.tile0[lo];
     return ti;
 }
 

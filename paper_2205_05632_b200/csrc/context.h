@@ -115,6 +115,7 @@ struct compams_context {
     int64_t W = 0;
 
     compams::Tables tab{};
+    compams::SegParams segp{};  // kernel-argument copy of the tiled blocks (nseg = 0: not usable)
     compams::BsBuffers bs{};
     compams::TopkBuffers tk{};
     int32_t* sel_small = nullptr;  // tiled blocks whose candidate lists one CTA selects from

@@ -149,10 +149,11 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const float* __restrict__ G) {
+__global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const float* __restrict__ G,
+                                                                 const __grid_constant__ SegParams sp_) {
     __shared__ uint2 sh_cand[kTileCand];
     __shared__ uint32_t sh_cnt, sh_base;
-    const TileInfo ti = load_tile(t.tiles, blockIdx.x);
+    const TileInfo ti = sp_.nseg ? find_tile(sp_, blockIdx.x) : load_tile(t.tiles, blockIdx.x);
     const int i = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const size_t sg = (size_t)i * t.nseg + ti.seg;
@@ -919,7 +920,7 @@ cudaError_t launch_topk_small(compams_context* c, const float* grads) {
 
 cudaError_t launch_topk_sweep(compams_context* c, const float* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    topk_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, grads);
+    topk_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, grads, c->segp);
     return cudaGetLastError();
 }
 
