@@ -201,3 +201,68 @@ def test_config4_resnet50_shapes_layerwise(comp):
 def test_config5_sweep_points_oracle_sized(mode, n):
     from parity import run_workload
     run_workload(W.sweep_point(1 << 20, n, mode, "cuda"), steps=3)
+
+
+# ------------------------------------------------------------------ the candidate path and its fallbacks
+
+def _status(opt):
+    return opt.buffer("status").cpu().tolist()
+
+
+def test_topk_candidate_path_is_taken_in_steady_state():
+    # after the first steps the threshold prediction must carry the selection: the dense passes stop
+    from parity import Pair
+    n, d = 4, 40 * 8192 + 321
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    p = Pair(n, d, [0, d], TOPK, 0.01)
+    try:
+        p.start(torch.zeros(d, device="cuda"))
+        for t in range(8):
+            p.step(torch.randn(n, d, generator=gen, device="cuda"), check_e=(t % 3 == 0))
+        st = _status(p.gpu)
+        assert st[0] == 0
+        assert st[1] + st[2] == 8 * n
+        assert st[1] <= 3 * n, "dense passes ran on %d of %d selections" % (st[1], 8 * n)
+    finally:
+        p.close()
+
+
+def test_topk_prediction_failures_fall_back_exactly():
+    # the gradient scale jumps by orders of magnitude between steps: too few candidates, too many,
+    # thresholds far above the predicted range - every case must still give the exact Top-k
+    scales = [1.0, 1.0, 1.0, 1.0, 300.0, 1.0, 1.0, 1e-3, 1e-3, 50.0, 1.0, 1.0]
+    n, d = 3, 25 * 8192 + 77
+    def make(gen, t):
+        return scales[t] * torch.randn(n, d, generator=gen, device="cuda")
+    _pair_run(n, d, [0, 6000, d], TOPK, 0.01, make, steps=len(scales), check_e_every=2)
+
+
+def test_topk_candidate_path_with_heavily_duplicated_values():
+    # a tiny alphabet: thousands of candidates share the threshold key, which neither the candidate
+    # list's threshold bin nor a plain radix pass can separate without the index order
+    n, d = 2, 30 * 8192
+    def make(gen, t):
+        return torch.randint(-20, 21, (n, d), generator=gen, device="cuda").float()
+    _pair_run(n, d, [0, d], TOPK, 0.01, make, steps=6, check_e_every=2)
+
+
+def test_topk_layerwise_many_lists_single_cta_select():
+    # many long candidate lists at once: the select runs one CTA per list instead of clusters
+    n = 8
+    offs = [0] + [int(x) for x in np.cumsum([120000] * 9)]
+    d = offs[-1]
+    _pair_run(n, d, offs, TOPK, 0.03, _randn(n, d), steps=5, check_e_every=2)
+
+
+def test_set_lr_takes_effect_on_the_next_step():
+    d = 5000
+    opt = CompAMS(2, d, [0, d], BLOCKSIGN)
+    theta = torch.zeros(d, device="cuda")
+    G = torch.randn(2, d, device="cuda")
+    opt.step(G, theta)
+    moved = theta.clone()
+    assert moved.abs().max() > 0
+    opt.set_lr(0.0)
+    opt.step(G, theta)
+    assert torch.equal(theta, moved)
+    opt.close()
