@@ -142,6 +142,15 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
         RC(dev_upload(c, &c->sel_big, big_l));
         c->n_sel_small = (int)small_l.size();
         c->n_sel_big = (int)big_l.size();
+        if (c->n_sel_big > 0) {
+            // enough slices for about four CTAs per SM over all long lists
+            const int64_t lists = (int64_t)c->n * c->n_sel_big;
+            int64_t parts = (4 * (int64_t)c->num_sms + lists - 1) / lists;
+            c->sel_parts = (int)(parts < 1 ? 1 : parts > 64 ? 64 : parts);
+            RC(dev_alloc(c, &c->tk.sel_hist, (size_t)lists * kSelBins));
+            RC(dev_alloc(c, &c->tk.sel_ticket, (size_t)lists * 2));
+            RC(dev_alloc(c, &c->tk.sel_surv, (size_t)lists * kSurvCap, false));
+        }
     }
     return COMPAMS_OK;
 }

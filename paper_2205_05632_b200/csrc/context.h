@@ -19,7 +19,7 @@ constexpr int kMaxTimed = 4096;    // event pairs kept for per-kernel timing
 
 constexpr uint32_t kNoPrediction = 0xffffffffu;  // tau_hat value that no key reaches
 constexpr int kTileCand = 1024;          // candidates one tile can stage in shared memory
-constexpr int kSelectCluster = 8;        // CTAs cooperating on one long candidate list
+constexpr int kSurvCap = 1536;           // threshold-bin candidates a select can rank in shared memory
 constexpr int kSelBins = 4096;           // bins of the candidate select's first histogram
 constexpr int kSelectSingleMax = 24576;  // candidate capacity up to which one CTA handles a segment
 
@@ -40,7 +40,8 @@ struct SegState {
     uint32_t ties_take;   // how many of them belong to the kept set
     uint32_t need_order;  // 1 when ties_take < ties_total: the lowest indices must be chosen
     uint32_t emit_count;  // message slots handed out so far
-    uint32_t pad[3];
+    uint32_t sel_ready;   // multi-CTA select: the threshold bin has been found, the emit kernel may run
+    uint32_t pad[2];
 };
 
 // Block / tile tables shared by the tiled kernels (device pointers).
@@ -80,6 +81,9 @@ struct TopkBuffers {
     uint2* cand;               // [n, cand_total] (coordinate, bits of x) pairs collected by the sweep
     int64_t cand_total;        // candidate slots per worker
     uint32_t* dense_count;     // [1] segments currently marked for the dense passes
+    uint32_t* sel_hist;        // [n * long lists, kSelBins] histogram a long list's slices add into
+    uint32_t* sel_ticket;      // [n * long lists, 2] slices arrived; threshold-bin candidates appended
+    uint2* sel_surv;           // [n * long lists, kSurvCap] threshold-bin candidates of a long list
     double* acc;               // [d] binary64 accumulator, used only by entries that overflow their bucket
     const uint32_t* kept_prev; // [n, map_words] bit j of row i: coordinate j was kept last step and its e is still
                                // to be zeroed (null when E is up to date)
@@ -121,6 +125,7 @@ struct compams_context {
     int32_t* sel_small = nullptr;  // tiled blocks whose candidate lists one CTA selects from
     int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists a cluster selects from
     int n_sel_small = 0, n_sel_big = 0;
+    int sel_parts = 1;  // slices a long candidate list is cut into
     uint32_t* keptmap[2] = {nullptr, nullptr};  // Top-k: kept maps of this and the previous step
     int map_cur = 0;
     bool e_mask_pending = false;  // Top-k: E still holds x at the coordinates kept in the last step

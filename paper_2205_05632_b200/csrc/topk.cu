@@ -11,13 +11,14 @@
 //   Candidate path (one pass over [n, d]):
 //     topk_sweep    x = g + e written over E (Algorithm 2, line 7); every key >= tau_hat, a threshold
 //                   predicted from the previous step, is appended to the segment's candidate list
-//     topk_select   one CTA (short lists) or a cluster of 8 CTAs (long lists) per segment: if the list
-//                   holds at least k_b and at most its capacity, the exact Top-k is inside it. A
-//                   histogram of the key offsets above tau_hat (bins sized from the last step, merged
-//                   through distributed shared memory) finds the threshold bin; winners above it are
-//                   emitted, the bin's few candidates go to rank 0's shared memory, which orders them
-//                   by (key, lower index first), keeps the best and predicts the next tau_hat.
-//                   Otherwise the segment is marked for the dense passes.
+//     topk_select   if the list holds at least k_b and at most its capacity, the exact Top-k is inside it.
+//                   A histogram of the key offsets above tau_hat (bins sized from the last step) finds
+//                   the threshold bin; winners above it are emitted, the bin's few candidates are
+//                   ordered by (key, lower index first), the best kept, and the next tau_hat predicted.
+//                   Otherwise the segment is marked for the dense passes. Short lists: one 1024-thread
+//                   CTA per list (topk_select). A few long lists (whole-vector selection): every list
+//                   is cut into slices handled by two kernels of ordinary CTAs (topk_selhist, topk_selemit)
+//                   that meet through a global histogram and last-slice-finishes tickets.
 //   Dense passes (only for marked segments; exact for any input, e.g. all-equal values), one
 //   cooperative kernel topk_dense whose stages are separated by grid-wide barriers:
 //     hist<1..3> / find<1..3>  three histogram passes over x, 11 + 10 + 10 key bits
@@ -185,7 +186,7 @@ __global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkB
 }
 
 // ------------------------------------------------------------------------------------------
-// select: exact Top-k inside the candidate list, one CTA or one cluster of CTAs per segment
+// select: exact Top-k inside the candidate list
 
 // Prediction for the next step's sweep, from this step's threshold key `tau` and the bin edge
 // `edge` at or above which about 2.5 k_b keys lay: the threshold keeps rising while the error
@@ -206,7 +207,6 @@ __device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_
     st->tau_prev = tau;
 }
 
-constexpr int kSurvCap = 1536;  // threshold-bin candidates one CTA can keep in shared memory
 constexpr int kSelUnroll = 4;   // candidate loads in flight per thread while scanning a list
 constexpr int kSelThreads = 1024;  // a select CTA is alone on its SM: many threads keep enough loads in flight
 constexpr int kSelWarps = kSelThreads / 32;
@@ -228,23 +228,25 @@ __device__ __forceinline__ uint32_t warp_slot(bool pred, uint32_t* counter, int 
 struct BinScan {
     uint32_t incl, excl;
 };
+template <int NT = kSelThreads>
 __device__ __forceinline__ BinScan scan_from_top(const uint32_t* hm, int nb, uint32_t* scratch, uint32_t* total) {
-    const int per = nb / kSelThreads > 0 ? nb / kSelThreads : 1;
+    const int per = nb / NT > 0 ? nb / NT : 1;
     uint32_t sum = 0;
     for (int j = 0; j < per; ++j) {
         const int bin = nb - 1 - ((int)threadIdx.x * per + j);
         if (bin >= 0) sum += hm[bin];
     }
     BinScan r;
-    r.incl = block_inclusive_scan<kSelWarps>(sum, scratch, total);
+    r.incl = block_inclusive_scan<NT / 32>(sum, scratch, total);
     r.excl = r.incl - sum;
     return r;
 }
 // The thread whose bins hold the `target`-th entry from the top writes
 // sh_out[0] = bin, sh_out[1] = entries above the bin, sh_out[2] = entries in the bin.
+template <int NT = kSelThreads>
 __device__ __forceinline__ void locate(const uint32_t* hm, int nb, const BinScan& sc, uint32_t target, uint32_t* sh_out) {
     if (sc.excl < target && target <= sc.incl) {
-        const int per = nb / kSelThreads > 0 ? nb / kSelThreads : 1;
+        const int per = nb / NT > 0 ? nb / NT : 1;
         uint32_t running = sc.excl;
         for (int j = 0; j < per; ++j) {
             const int bin = nb - 1 - ((int)threadIdx.x * per + j);
@@ -259,18 +261,19 @@ __device__ __forceinline__ void locate(const uint32_t* hm, int nb, const BinScan
     }
 }
 
+__device__ __forceinline__ uint32_t offset_digit(uint32_t xbits, uint32_t tau_hat, int S) {
+    const uint32_t dg = ((xbits & 0x7fffffffu) - tau_hat) >> S;  // every candidate has key >= tau_hat
+    return dg < (uint32_t)(kSelBins - 1) ? dg : (uint32_t)(kSelBins - 1);
+}
+
 __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                int nlist) {
-    __shared__ uint32_t local[kSelBins];   // this CTA's histogram
-    __shared__ uint32_t merged[kSelBins];  // rank 0's copy receives every CTA's counts
+    __shared__ uint32_t local[kSelBins];  // histogram of the list
     __shared__ uint2 surv[kSurvCap];
     __shared__ uint32_t scratch[kSelWarps];
     __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt;
-    cg::cluster_group cluster = cg::this_cluster();
-    const unsigned rank = cluster.block_rank();
-    const unsigned nrank = cluster.num_blocks();
     const int lane = threadIdx.x & 31;
-    const size_t item = blockIdx.x / nrank;
+    const size_t item = blockIdx.x;
     const int i = (int)(item / (size_t)nlist);
     const int seg = seg_list[item % (size_t)nlist];
     const size_t sg = (size_t)i * t.nseg + seg;
@@ -280,32 +283,21 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
     const uint32_t c = st->cand_count;
     const uint32_t tau_hat = st->tau_hat;
     const int S = (int)st->sel_shift;
-    // the same decision in every CTA of the cluster: they read the same words and nobody writes them here
     if (!(tau_hat != kNoPrediction && c >= kb && c <= cap)) {
-        if (rank == 0 && threadIdx.x == 0) {
+        if (threadIdx.x == 0) {
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
         }
         return;
     }
-    uint32_t* merged0 = cluster.map_shared_rank(&merged[0], 0);
     const uint2* list = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
-    const uint32_t per = (c + nrank - 1) / nrank;
-    const uint32_t lo = rank * per;
-    const uint32_t hi = (lo + per < c) ? lo + per : c;
-    auto digit0 = [&](uint32_t xbits) -> uint32_t {
-        const uint32_t o = (xbits & 0x7fffffffu) - tau_hat;  // every candidate has key >= tau_hat
-        const uint32_t dg = o >> S;
-        return dg < (uint32_t)(kSelBins - 1) ? dg : (uint32_t)(kSelBins - 1);
-    };
+    const uint32_t lo = 0u, hi = c;
+    auto digit0 = [&](uint32_t xbits) -> uint32_t { return offset_digit(xbits, tau_hat, S); };
 
     // ---- pass 0: histogram of the key offsets above tau_hat in bins of 2^S; the last bin is open-ended
-    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads) {
-        local[k] = 0u;
-        merged[k] = 0u;
-    }
+    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads) local[k] = 0u;
     if (threadIdx.x == 0) sh_scnt = 0u;
-    cluster.sync();
+    __syncthreads();
     for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kSelThreads) {
         uint32_t y[kSelUnroll];
 #pragma unroll
@@ -325,19 +317,14 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
         }
     }
     __syncthreads();
-    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads) {
-        const uint32_t v = local[k];
-        if (v) atomicAdd(merged0 + k, v);
-    }
-    cluster.sync();
     uint32_t total;
     {
-        const BinScan sc = scan_from_top(merged0, kSelBins, scratch, &total);
+        const BinScan sc = scan_from_top(local, kSelBins, scratch, &total);
         const uint32_t want = 2u * kb + (kb >> 1);
         if (threadIdx.x == 0) sh_edge[0] = 0xffffffffu;  // "fewer than `want` candidates"
         __syncthreads();
-        locate(merged0, kSelBins, sc, kb, sh_bin);
-        locate(merged0, kSelBins, sc, want, sh_edge);
+        locate(local, kSelBins, sc, kb, sh_bin);
+        locate(local, kSelBins, sc, want, sh_edge);
     }
     __syncthreads();
     const uint32_t b0 = sh_bin[0];
@@ -345,26 +332,26 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
     const uint32_t c0 = sh_bin[2];
     const uint32_t edge_bin = sh_edge[0];
     const bool take_all0 = (c0 == k_rem);
-    // this CTA's own share of the winners, from its private histogram
+    // the number of winners, from the histogram
     uint32_t mine = 0;
     for (int k = threadIdx.x; k < kSelBins; k += kSelThreads)
         if ((uint32_t)k > b0 || (take_all0 && (uint32_t)k == b0)) mine += local[k];
     uint32_t my_winners;
     block_inclusive_scan<kSelWarps>(mine, scratch, &my_winners);
-    cluster.sync();  // everybody has read rank 0's histogram
+    __syncthreads();
     if (b0 == (uint32_t)(kSelBins - 1) && !take_all0) {
         // the threshold lies in the open-ended bin: the prediction was far off, let the dense passes decide
-        if (rank == 0 && threadIdx.x == 0) {
+        if (threadIdx.x == 0) {
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
         }
         return;
     }
 
-    // ---- second scan of the list: winners to the message, threshold-bin candidates to rank 0's shared memory
+    // ---- second scan of the list: winners to the message, threshold-bin candidates to shared memory
     const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
-    uint2* surv0 = cluster.map_shared_rank(&surv[0], 0);
-    uint32_t* scnt0 = cluster.map_shared_rank(&sh_scnt, 0);
+    uint2* surv0 = &surv[0];
+    uint32_t* scnt0 = &sh_scnt;
     if (threadIdx.x == 0) {
         sh_base = my_winners ? atomicAdd(&st->emit_count, my_winners) : 0u;
         sh_wcnt = 0u;
@@ -403,8 +390,7 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
     const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
     uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
     if (!take_all0) {
-        cluster.sync();  // every CTA's threshold-bin candidates have reached rank 0
-        if (rank != 0) return;
+        __syncthreads();
         const uint32_t nsurv = sh_scnt;
         if (nsurv > (uint32_t)kSurvCap) {
             // too many candidates share the threshold bin (heavily duplicated values): dense passes
@@ -414,7 +400,7 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
             }
             return;
         }
-        // ---- rank 0 orders the survivors by (key, lower index first): survivor q is kept when fewer
+        // ---- the survivors are ordered by (key, lower index first): survivor q is kept when fewer
         // than k_rem survivors beat it
         const uint32_t lowmask = S ? ((1u << S) - 1u) : 0u;
         auto comp_of = [&](const uint2& cv) -> unsigned long long {
@@ -450,7 +436,260 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
         }
         tau = sh_edge[1];
     }
-    if (rank == 0 && threadIdx.x == 0) {
+    if (threadIdx.x == 0) {
+        uint32_t edge;
+        if (edge_bin != 0xffffffffu) {
+            const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
+            edge = ew < 0x7f7fffffull ? (uint32_t)ew : 0x7f7fffffu;
+        } else {
+            // fewer than 2.5 k_b candidates: reach further down next time, by half the distance to the threshold
+            const uint32_t gap = ((tau - tau_hat) >> 1) + (1u << 16);
+            edge = tau_hat > gap ? tau_hat - gap : 0u;
+        }
+        predict_next(st, tau, edge, true);
+        st->fallback = 0u;
+        atomicAdd(b.status + 2, 1u);  // selections decided inside their candidate list
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// select for a few long lists (whole-vector selection): every list is cut into `parts` slices and
+// two kernels of ordinary CTAs work on all slices at once. The slices of a list meet through a
+// histogram in global memory and "the last slice to arrive does the serial part" tickets; nobody
+// waits for anybody.
+//   topk_selhist  slice histograms of the key offsets above tau_hat, added into the list's global
+//                 histogram; the last slice finds the threshold bin and the next tau_hat's bin edge
+//   topk_selemit  winners above the threshold bin go to the message, the bin's candidates to the
+//                 list's survivor buffer; the last slice ranks the survivors, emits the best and predicts
+
+__global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
+                                                                int nlist, int parts) {
+    __shared__ uint32_t local[kSelBins];
+    __shared__ uint32_t scratch[kWarps];
+    __shared__ uint32_t sh_bin[3], sh_edge[3];
+    __shared__ int is_last;
+    const int lane = threadIdx.x & 31;
+    const int part = blockIdx.x % parts;
+    const size_t item = blockIdx.x / parts;  // (worker, list)
+    const int i = (int)(item / (size_t)nlist);
+    const int seg = seg_list[item % (size_t)nlist];
+    const size_t sg = (size_t)i * t.nseg + seg;
+    const SegInfo* si = t.segs + seg;
+    SegState* st = b.seg + sg;
+    const uint32_t kb = si->kb, cap = si->cap;
+    const uint32_t c = st->cand_count;
+    const uint32_t tau_hat = st->tau_hat;
+    const int S = (int)st->sel_shift;
+    // the same decision in every slice of the list: nobody writes these words in this kernel
+    if (!(tau_hat != kNoPrediction && c >= kb && c <= cap)) {
+        if (part == 0 && threadIdx.x == 0) {
+            st->fallback = 1u;
+            atomicAdd(b.dense_count, 1u);
+        }
+        return;
+    }
+    const uint2* list = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
+    const uint32_t per = (c + parts - 1) / parts;
+    const uint32_t lo = (uint32_t)part * per < c ? (uint32_t)part * per : c;
+    const uint32_t hi = (lo + per < c) ? lo + per : c;
+    for (int k = threadIdx.x; k < kSelBins; k += kThreads) local[k] = 0u;
+    __syncthreads();
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+        uint32_t y[kSelUnroll];
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const uint32_t p = p0 + u * kThreads + threadIdx.x;
+            y[u] = p < hi ? list[p].y : 0xffffffffu;  // no candidate has this pattern (NaN)
+        }
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const bool valid = y[u] != 0xffffffffu;
+            const uint32_t dg = valid ? offset_digit(y[u], tau_hat, S) : 0u;
+            // the open-ended last bin collects every far-above-threshold candidate: one atomic per warp
+            const bool far = valid && dg == (uint32_t)(kSelBins - 1);
+            const unsigned m = __ballot_sync(0xffffffffu, far);
+            if (m && lane == __ffs(m) - 1) atomicAdd(&local[kSelBins - 1], (uint32_t)__popc(m));
+            if (valid && !far) atomicAdd(&local[dg], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t* gh = b.sel_hist + item * kSelBins;
+    for (int k = threadIdx.x; k < kSelBins; k += kThreads) {
+        const uint32_t v = local[k];
+        if (v) atomicAdd(gh + k, v);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(b.sel_ticket + 2 * item, 1u) == (uint32_t)(parts - 1));
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    // ---- the last slice: the list's histogram is complete
+    for (int k = threadIdx.x; k < kSelBins; k += kThreads) {
+        local[k] = __ldcg(gh + k);
+        gh[k] = 0u;  // clean for the next step
+    }
+    __syncthreads();
+    uint32_t total;
+    const BinScan sc = scan_from_top<kThreads>(local, kSelBins, scratch, &total);
+    const uint32_t want = 2u * kb + (kb >> 1);
+    if (threadIdx.x == 0) sh_edge[0] = 0xffffffffu;  // "fewer than `want` candidates"
+    __syncthreads();
+    locate<kThreads>(local, kSelBins, sc, kb, sh_bin);
+    locate<kThreads>(local, kSelBins, sc, want, sh_edge);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        b.sel_ticket[2 * item] = 0u;
+        const uint32_t b0 = sh_bin[0], k_rem = kb - sh_bin[1];
+        const bool take_all0 = (sh_bin[2] == k_rem);
+        if (b0 == (uint32_t)(kSelBins - 1) && !take_all0) {
+            // the threshold lies in the open-ended bin: the prediction was far off, let the dense passes decide
+            st->fallback = 1u;
+            atomicAdd(b.dense_count, 1u);
+        } else {
+            st->prefix = b0;  // the dense passes' fields are free while the candidate path owns the segment
+            st->k_rem = k_rem;
+            st->ties_total = take_all0 ? 1u : 0u;
+            st->edge = sh_edge[0];
+            st->sel_ready = 1u;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
+                                                                int nlist, int parts) {
+    __shared__ uint2 surv[kSurvCap];
+    __shared__ uint32_t scratch[kWarps];
+    __shared__ uint32_t sh_base, sh_wcnt, sh_tau;
+    __shared__ int is_last;
+    const int lane = threadIdx.x & 31;
+    const int part = blockIdx.x % parts;
+    const size_t item = blockIdx.x / parts;
+    const int i = (int)(item / (size_t)nlist);
+    const int seg = seg_list[item % (size_t)nlist];
+    const size_t sg = (size_t)i * t.nseg + seg;
+    const SegInfo* si = t.segs + seg;
+    SegState* st = b.seg + sg;
+    if (st->sel_ready == 0u) return;  // not decided by the candidate path (same word for every slice)
+    const uint32_t kb = si->kb;
+    const uint32_t c = st->cand_count;
+    const uint32_t tau_hat = st->tau_hat;
+    const int S = (int)st->sel_shift;
+    const uint32_t b0 = st->prefix, k_rem = st->k_rem, edge_bin = st->edge;
+    const bool take_all0 = st->ties_total != 0u;
+    const uint2* list = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
+    const uint32_t per = (c + parts - 1) / parts;
+    const uint32_t lo = (uint32_t)part * per < c ? (uint32_t)part * per : c;
+    const uint32_t hi = (lo + per < c) ? lo + per : c;
+    const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
+    uint2* gsurv = b.sel_surv + item * kSurvCap;
+    uint32_t* gscnt = b.sel_ticket + 2 * item + 1;  // survivors appended so far (second word of the pair)
+
+    // first pass over the slice (from L2): how many winners, so that they get one contiguous slot range
+    uint32_t mine = 0;
+    for (uint32_t p = lo + threadIdx.x; p < hi; p += kThreads) {
+        const uint32_t dg = offset_digit(list[p].y, tau_hat, S);
+        mine += (dg > b0 || (take_all0 && dg == b0)) ? 1u : 0u;
+    }
+    uint32_t my_winners;
+    block_inclusive_scan(mine, scratch, &my_winners);
+    if (threadIdx.x == 0) {
+        sh_base = my_winners ? atomicAdd(&st->emit_count, my_winners) : 0u;
+        sh_wcnt = 0u;
+    }
+    __syncthreads();
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+        uint2 cvs[kSelUnroll];
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const uint32_t p = p0 + u * kThreads + threadIdx.x;
+            cvs[u] = p < hi ? list[p] : make_uint2(0u, 0xffffffffu);
+        }
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            const uint2 cv = cvs[u];
+            const bool valid = cv.y != 0xffffffffu;
+            const uint32_t dg = valid ? offset_digit(cv.y, tau_hat, S) : 0u;
+            const bool win = valid && (dg > b0 || (take_all0 && dg == b0));
+            const bool keep = valid && !take_all0 && dg == b0;
+            const uint32_t wpos = sh_base + warp_slot(win, &sh_wcnt, lane);
+            if (win) {
+                if (wpos < kb) {
+                    b.idx[slot0 + wpos] = (int32_t)cv.x;
+                    b.val[slot0 + wpos] = __uint_as_float(cv.y);
+                } else {
+                    atomicOr(b.status, 1u);
+                }
+            }
+            if (__any_sync(0xffffffffu, keep)) {  // rare: only the threshold bin's candidates
+                const uint32_t spos = warp_slot(keep, gscnt, lane);
+                if (keep && spos < (uint32_t)kSurvCap) gsurv[spos] = cv;
+            }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(b.sel_ticket + 2 * item, 1u) == (uint32_t)(parts - 1));
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    // ---- the last slice finishes the list
+    const uint32_t nsurv = take_all0 ? 0u : __ldcg(gscnt);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        b.sel_ticket[2 * item] = 0u;
+        b.sel_ticket[2 * item + 1] = 0u;
+        st->sel_ready = 0u;
+    }
+    if (nsurv > (uint32_t)kSurvCap) {
+        // too many candidates share the threshold bin (heavily duplicated values): dense passes
+        if (threadIdx.x == 0) {
+            st->fallback = 1u;
+            atomicAdd(b.dense_count, 1u);
+        }
+        return;
+    }
+    const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
+    uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
+    if (!take_all0) {
+        for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) surv[q] = __ldcg(gsurv + q);
+        __syncthreads();
+        // survivor q is kept when fewer than k_rem survivors beat it in (key, lower index first) order
+        const uint32_t lowmask = S ? ((1u << S) - 1u) : 0u;
+        auto comp_of = [&](const uint2& cv) -> unsigned long long {
+            const uint32_t o = (cv.y & 0x7fffffffu) - tau_hat;
+            return ((unsigned long long)(o & lowmask) << 32) | (unsigned long long)(0xffffffffu - cv.x);
+        };
+        for (uint32_t q0 = 0; q0 < nsurv; q0 += kThreads) {  // uniform trip count: the loop holds barriers
+            const uint32_t q = q0 + threadIdx.x;
+            bool kept = false;
+            uint2 cv = make_uint2(0u, 0u);
+            if (q < nsurv) {
+                cv = surv[q];
+                const unsigned long long mine_c = comp_of(cv);
+                uint32_t beaten = 0;
+                for (uint32_t p = 0; p < nsurv; ++p) beaten += (comp_of(surv[p]) > mine_c) ? 1u : 0u;
+                kept = beaten < k_rem;
+                if (beaten == k_rem - 1u) sh_tau = (cv.y & 0x7fffffffu);  // the k-th largest key overall
+            }
+            uint32_t tot3;
+            const uint32_t incl = block_inclusive_scan(kept ? 1u : 0u, scratch, &tot3);
+            if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
+            __syncthreads();
+            if (kept) {
+                const uint32_t pos = sh_base + incl - 1u;
+                if (pos < kb) {
+                    b.idx[slot0 + pos] = (int32_t)cv.x;
+                    b.val[slot0 + pos] = __uint_as_float(cv.y);
+                } else {
+                    atomicOr(b.status, 1u);
+                }
+            }
+            __syncthreads();
+        }
+        tau = sh_tau;
+    }
+    if (threadIdx.x == 0) {
         uint32_t edge;
         if (edge_bin != 0xffffffffu) {
             const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
@@ -924,28 +1163,20 @@ cudaError_t launch_topk_sweep(compams_context* c, const float* grads) {
     return cudaGetLastError();
 }
 
-// One launch per list of segments: short candidate lists get one CTA each, long ones a cluster.
-static cudaError_t launch_select_list(compams_context* c, const int32_t* list, int nlist, int cluster) {
-    if (nlist == 0) return cudaSuccess;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((int64_t)c->n * nlist * cluster), 1, 1);
-    cfg.blockDim = dim3(kSelThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = c->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)cluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, topk_select_kernel, c->tab, c->tk, list, nlist);
-}
-
 cudaError_t launch_topk_select(compams_context* c) {
-    cudaError_t e = launch_select_list(c, c->sel_small, c->n_sel_small, 1);
+    cudaError_t e = cudaSuccess;
+    if (c->n_sel_small > 0) {
+        topk_select_kernel<<<(unsigned)((int64_t)c->n * c->n_sel_small), kSelThreads, 0, c->stream>>>(
+            c->tab, c->tk, c->sel_small, c->n_sel_small);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess || c->n_sel_big == 0) return e;
+    const unsigned grid = (unsigned)((int64_t)c->n * c->n_sel_big * c->sel_parts);
+    topk_selhist_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, c->sel_big, c->n_sel_big, c->sel_parts);
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return launch_select_list(c, c->sel_big, c->n_sel_big, kSelectCluster);
+    topk_selemit_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, c->sel_big, c->n_sel_big, c->sel_parts);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_topk_dense(compams_context* c) {
