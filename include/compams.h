@@ -64,9 +64,12 @@ enum compams_buffer {
     COMPAMS_BUF_SIGN_BITS = 8,    /* uint32 [n, W]   Block-Sign sign bits, see below; W = sum_b ceil(d_b / 32)   */
     COMPAMS_BUF_SIGN_WORD_OFFSETS = 9, /* int64 [M+1] first word of block b inside a row of SIGN_BITS            */
     COMPAMS_BUF_SCALES = 10,      /* float  [n, M]   Block-Sign scales ||x_B||_1 / d_B                           */
-    COMPAMS_BUF_STATUS = 11       /* uint32 [4]      [0] status word (0 = clean); Top-k counters since creation:
+    COMPAMS_BUF_STATUS = 11       /* uint32 [8]      [0] status word (0 = clean); Top-k counters since creation:
                                                     [1] (worker, block) selections done by the dense passes,
-                                                    [2] selections done inside the candidate list; [3] unused  */
+                                                    [2] selections done inside the candidate list; why a list
+                                                    was given up: [3] fewer candidates than k_b, [4] more than
+                                                    its capacity, [5] threshold beyond the histogram's range,
+                                                    [6] too many candidates sharing the threshold bin; [7] unused */
 };
 
 /* Kernel identifiers for compams_get_kernel_time. */

@@ -171,7 +171,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
     RC(dev_alloc(c, &c->v, (size_t)d));
     RC(dev_alloc(c, &c->vhat, (size_t)d));
     RC(dev_alloc(c, &c->gbar, (size_t)d));
-    RC(dev_alloc(c, &c->status, 4));
+    RC(dev_alloc(c, &c->status, 8));
 
     if (c->compressor == COMPAMS_TOPK) {
         c->seg_off.assign((size_t)M + 1, 0);
@@ -469,7 +469,7 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
         case COMPAMS_BUF_SIGN_BITS: if (sign) { p = c->bs.bits; cnt = (int64_t)c->n * c->W; } break;
         case COMPAMS_BUF_SIGN_WORD_OFFSETS: if (sign) { p = c->d_word_off; cnt = c->M + 1; } break;
         case COMPAMS_BUF_SCALES: if (sign) { p = c->scales[c->scales_cur]; cnt = (int64_t)c->n * c->M; } break;
-        case COMPAMS_BUF_STATUS: p = c->status; cnt = 4; break;
+        case COMPAMS_BUF_STATUS: p = c->status; cnt = 8; break;
         default: return COMPAMS_ERR_INVALID_ARG;
     }
     *dev_ptr = p;

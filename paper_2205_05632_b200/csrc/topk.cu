@@ -287,6 +287,7 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
         if (threadIdx.x == 0) {
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
+            if (tau_hat != kNoPrediction) atomicAdd(b.status + (c < kb ? 3 : 4), 1u);  // too few / too many candidates
         }
         return;
     }
@@ -344,6 +345,7 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
         if (threadIdx.x == 0) {
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
+            atomicAdd(b.status + 5, 1u);
         }
         return;
     }
@@ -397,6 +399,7 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
             if (threadIdx.x == 0) {
                 st->fallback = 1u;
                 atomicAdd(b.dense_count, 1u);
+                atomicAdd(b.status + 6, 1u);
             }
             return;
         }
@@ -485,6 +488,7 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
         if (part == 0 && threadIdx.x == 0) {
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
+            if (tau_hat != kNoPrediction) atomicAdd(b.status + (c < kb ? 3 : 4), 1u);  // too few / too many candidates
         }
         return;
     }
@@ -546,6 +550,7 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
             // the threshold lies in the open-ended bin: the prediction was far off, let the dense passes decide
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
+            atomicAdd(b.status + 5, 1u);
         } else {
             st->prefix = b0;  // the dense passes' fields are free while the candidate path owns the segment
             st->k_rem = k_rem;
@@ -646,6 +651,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
         if (threadIdx.x == 0) {
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
+            atomicAdd(b.status + 6, 1u);
         }
         return;
     }
