@@ -1,5 +1,6 @@
 // C ABI of the COMP-AMS library (see include/compams.h): argument checks, state allocation,
 // the per-step launch sequence and the inspection calls.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -72,7 +73,12 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
     for (size_t s = 0; s < blocks.size(); ++s) {
         const int32_t b = blocks[s];
         const int64_t len = c->off[b + 1] - c->off[b];
-        const int64_t nt = (len + kTile - 1) / kTile;
+        // The sweeps shift a worker's tiles down by the phase of the block's first element within a
+        // 128-byte line, (i d + o) mod 32, so that every warp access covers whole lines; the block
+        // needs enough tiles for the largest shift among the workers.
+        int64_t smax = 0;
+        for (int32_t i = 0; i < c->n && smax < 31; ++i) smax = std::max<int64_t>(smax, ((int64_t)i * c->d + c->off[b]) & 31);
+        const int64_t nt = (len + smax + kTile - 1) / kTile;
         if ((int64_t)tiles.size() + nt > (int64_t)0x7fffffff) return COMPAMS_ERR_INVALID_ARG;
         SegInfo si{};
         si.o = c->off[b];
@@ -91,7 +97,7 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
             si.cand_off = cand_total;
             cand_total += cap;
         }
-        for (int64_t r0 = 0; r0 < len; r0 += kTile) {
+        for (int64_t r0 = 0; r0 < nt * kTile; r0 += kTile) {
             TileInfo ti{};
             ti.o = c->off[b];
             ti.len = (int32_t)len;
@@ -222,9 +228,9 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &t.tile_ties, (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &t.cand, (size_t)n * (size_t)t.cand_total, false));
         RC(dev_alloc(c, &t.acc, (size_t)d));
-        t.map_words = (d + 31) / 32;
-        RC(dev_alloc(c, &c->keptmap[0], (size_t)n * (size_t)t.map_words));
-        RC(dev_alloc(c, &c->keptmap[1], (size_t)n * (size_t)t.map_words));
+        t.map_words = ((int64_t)n * d + 31) / 32;
+        RC(dev_alloc(c, &c->keptmap[0], (size_t)t.map_words));
+        RC(dev_alloc(c, &c->keptmap[1], (size_t)t.map_words));
         {
             // kept entries are handed to the server grouped by coordinate range: room for four times the
             // average load of a bucket, the rare excess goes through the binary64 accumulator
@@ -252,6 +258,8 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
             word_off[(size_t)b + 1] = word_off[(size_t)b] + (c->off[b + 1] - c->off[b] + 31) / 32;
         c->W = word_off[(size_t)M];
         RC(dev_upload(c, &c->d_word_off, word_off));
+        if (c->W > (int64_t)INT32_MAX) c->segp.nseg = 0;  // word offsets would not fit the kernel-argument copy
+        for (int32_t sg = 0; sg < c->segp.nseg; ++sg) c->segp.wofs[sg] = (int32_t)word_off[(size_t)c->segp.blk[sg]];
         BsBuffers& s = c->bs;
         s.E = c->E;
         s.word_off = c->d_word_off;
@@ -260,6 +268,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &c->scales[0], (size_t)n * (size_t)M));
         RC(dev_alloc(c, &c->scales[1], (size_t)n * (size_t)M));
         RC(dev_alloc(c, &s.tile_sum, (size_t)n * (size_t)c->tab.ntiles));
+        RC(dev_alloc(c, &s.edge, (size_t)n * (size_t)c->tab.ntiles));
         s.gbar = c->gbar;
         s.m = c->m;
         s.v = c->v;
@@ -321,7 +330,7 @@ int step_device(compams_context* c, const float* grads, float* theta) {
     c->map_cur ^= 1;
     c->tk.kept_cur = c->keptmap[c->map_cur];
     c->tk.kept_prev = c->e_mask_pending ? c->keptmap[c->map_cur ^ 1] : nullptr;
-    CU(cudaMemsetAsync(c->tk.kept_cur, 0, (size_t)c->n * (size_t)c->tk.map_words * sizeof(uint32_t), c->stream));
+    CU(cudaMemsetAsync(c->tk.kept_cur, 0, (size_t)c->tk.map_words * sizeof(uint32_t), c->stream));
     if (c->tk.nsmall > 0) RC(run_kernel(c, COMPAMS_K_TOPK_SMALL, [&] { return launch_topk_small(c, grads); }));
     if (c->tab.ntiles > 0) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));

@@ -33,25 +33,28 @@ __device__ __forceinline__ double abs_as_double(float x) {
     return __hiloint2double((int)((b >> 3) + 0x38000000u), (int)(b << 29));
 }
 
+// One warp's 1024 consecutive coordinates starting at rw (relative to the block; rw may be negative
+// or reach past the block in a tile at either end of it: such coordinates are skipped).
 template <bool FULL>
 __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int rw,
-                                              int lane, bool deferred, float sp, double& acc, uint32_t& myword) {
-    const int cg = align_class(g), ce = align_class(e);
+                                              int lane, bool deferred, float sp, double& acc, uint32_t& mymask) {
+    const int cg = align_class(g + rw), ce = align_class(e + rw);
 #pragma unroll
     for (int bt = 0; bt < kIters / 2; ++bt) {
         float4 gv[2], ev[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int r = rw + (bt * 2 + u) * 128 + lane * 4;
-            if (FULL || r + 3 < len) {
+            if (FULL || (r >= 0 && r + 3 < len)) {
                 gv[u] = load4_stream(g + r, cg);
                 ev[u] = load4(e + r, ce);
             } else {
                 float gt[4], et[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    gt[k] = (r + k < len) ? __ldg(g + r + k) : 0.0f;
-                    et[k] = (r + k < len) ? e[r + k] : 0.0f;
+                    const bool live = (unsigned)(r + k) < (unsigned)len;
+                    gt[k] = live ? __ldg(g + r + k) : 0.0f;
+                    et[k] = live ? e[r + k] : 0.0f;
                 }
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
                 ev[u] = make_float4(et[0], et[1], et[2], et[3]);
@@ -70,52 +73,76 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
                 float ee = deferred ? __fsub_rn(xo, copysignf(sp, xo)) : xo;
                 float x = __fadd_rn(lane_elem(gv[u], k), ee);  // line 7: x = g + e
                 xs[k] = x;
-                const bool live = FULL || (r + k < len);
+                const bool live = FULL || ((unsigned)(r + k) < (unsigned)len);
                 if (live) {
                     acc += abs_as_double(x);
                     nib |= (__float_as_uint(x) >> 31) << k;
                 }
             }
-            if (FULL || r + 3 < len) {
+            if (FULL || (r >= 0 && r + 3 < len)) {
                 store4(e + r, ce, make_float4(xs[0], xs[1], xs[2], xs[3]));
             } else {
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    if (r + k < len) e[r + k] = xs[k];
+                    if ((unsigned)(r + k) < (unsigned)len) e[r + k] = xs[k];
             }
             uint32_t w = pack_group_word(nib, lane);
             uint32_t wv = __shfl_sync(0xffffffffu, w, (lane & 3) * 8);
-            if ((lane >> 2) == it) myword = wv;  // lane l ends up holding word l of the warp's 32 words
+            if ((lane >> 2) == it) mymask = wv;  // lane l ends up holding the sign mask of the warp's l-th 32 coordinates
         }
     }
 }
 
+// Tiles are shifted down by s = (i d + o) mod 32, the position of the block's first element within
+// a 128-byte line of G and E, so that every warp access covers whole lines (with rows that start
+// mid-line a warp's 512 bytes straddle five lines instead of four: measured 7 % slower). The
+// sign words stay indexed by coordinate: word q of the block takes its low 32 - s bits from the
+// q-th group of 32 shifted coordinates and its high s bits from the next group. The word a tile
+// shares with the next tile is put together by bs_scales from the two shares left in `edge`.
 __global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffers b, const float* __restrict__ G,
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
+    __shared__ uint32_t sh_first[kWarps];
     const int tile = blockIdx.x;
     const int i = blockIdx.y;
     const TileInfo ti = sp_.nseg ? find_tile(sp_, tile) : load_tile(t.tiles, tile);
     const int blk = ti.blk;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float* g = G + (size_t)i * (size_t)t.d + (size_t)ti.o;
-    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
+    const int64_t row0 = (int64_t)i * t.d + ti.o;
+    const int s = (int)(row0 & 31);
+    const float* g = G + row0;
+    float* e = b.E + row0;
     const float sp = deferred ? b.scales_prev[(size_t)i * t.M + blk] : 0.0f;
-    const int rw = ti.r0 + warp * kWarpSpan;
+    const int r0s = ti.r0 - s;
+    const int rw = r0s + warp * kWarpSpan;
 
     double acc = 0.0;
-    uint32_t myword = 0;
-    if (ti.r0 + kTile <= ti.len)
-        bs_sweep_tile<true>(g, e, ti.len, rw, lane, deferred != 0, sp, acc, myword);
+    uint32_t mymask = 0;
+    if (r0s >= 0 && r0s + kTile <= ti.len)
+        bs_sweep_tile<true>(g, e, ti.len, rw, lane, deferred != 0, sp, acc, mymask);
     else
-        bs_sweep_tile<false>(g, e, ti.len, rw, lane, deferred != 0, sp, acc, myword);
-
-    if (rw + lane * 32 < ti.len)
-        b.bits[(size_t)i * (size_t)b.W + (size_t)b.word_off[blk] + (size_t)(rw >> 5) + lane] = myword;
+        bs_sweep_tile<false>(g, e, ti.len, rw, lane, deferred != 0, sp, acc, mymask);
 
     // tile sum in binary64 (fixed shuffle tree); bs_scales adds the tile sums of a block in a fixed order
-    double s = block_sum_double(acc, red);
-    if (threadIdx.x == 0) b.tile_sum[(size_t)i * t.ntiles + tile] = s;
+    if (lane == 0) sh_first[warp] = mymask;
+    const double sum = block_sum_double(acc, red);  // its barriers also publish sh_first
+    if (threadIdx.x == 0) b.tile_sum[(size_t)i * t.ntiles + tile] = sum;
+
+    uint32_t next = __shfl_down_sync(0xffffffffu, mymask, 1);
+    const bool last = warp == kWarps - 1 && lane == 31;
+    if (lane == 31) next = last ? 0u : sh_first[warp + 1];
+    const uint32_t word = __funnelshift_r(mymask, next, (uint32_t)s);  // s = 0: the mask itself
+    const int q = (ti.r0 >> 5) + warp * 32 + lane;  // word of the block this lane completes
+    const int wb = (ti.len + 31) >> 5;
+    const int64_t wofs = sp_.nseg ? (int64_t)sp_.wofs[ti.seg] : b.word_off[blk];
+    if (!last && q < wb) b.bits[(size_t)i * (size_t)b.W + (size_t)wofs + (size_t)q] = word;
+    // shares of the two words in common with the neighbouring tiles: the high bits of the word before
+    // this tile's first, the low bits of its last
+    if (threadIdx.x == 0 || last) {
+        uint32_t* ed = reinterpret_cast<uint32_t*>(b.edge + (size_t)i * t.ntiles + tile);
+        if (last) ed[1] = word;
+        else ed[0] = s ? (mymask << (32 - s)) : 0u;
+    }
 }
 
 // One CTA per (worker, block): scale = ||x_B||_1 / d_B from the tile sums (Definition 2).
@@ -126,6 +153,16 @@ __global__ void __launch_bounds__(kThreads) bs_scales_kernel(Tables t, BsBuffers
     const double* ts = b.tile_sum + (size_t)i * t.ntiles + si->tile0;
     double part = 0.0;
     for (int k = threadIdx.x; k < si->ntile_b; k += kThreads) part += ts[k];
+    // the sign word two neighbouring tiles have in common: one share from each
+    {
+        const uint2* ed = b.edge + (size_t)i * t.ntiles + si->tile0;
+        const int wb = (si->len + 31) >> 5;
+        uint32_t* words = b.bits + (size_t)i * (size_t)b.W + (size_t)b.word_off[blk];
+        for (int k = threadIdx.x; k < si->ntile_b; k += kThreads) {
+            const int q = (k + 1) * (kTile / 32) - 1;
+            if (q < wb) words[q] = ed[k].y | (k + 1 < si->ntile_b ? ed[k + 1].x : 0u);
+        }
+    }
     const double S = block_sum_double(part, red);
     // one division in binary64, one rounding to fp32
     if (threadIdx.x == 0) b.scales_cur[(size_t)i * t.M + blk] = __double2float_rn(S / (double)si->len);
@@ -151,23 +188,43 @@ __global__ void __launch_bounds__(kThreads) bs_materialize_kernel(Tables t, floa
 
 constexpr int kApplyChunk = 64;  // workers whose sign words are staged in shared memory at a time
 
-// One CTA per 1024 consecutive coordinates of a block (one float4 group per thread).
-__global__ void __launch_bounds__(kThreads, 6) bs_apply_kernel(Tables t, BsBuffers b, float* __restrict__ theta,
-                                                               HyperParams hp) {
+// Server side of Block-Sign (Algorithm 2, lines 12-16): one CTA per 1024 consecutive coordinates of a
+// block, one float4 group per thread. The tile's block comes from the constant bank, so the sign
+// words, the scales and the optimizer state are all requested at once. Per coordinate the sum over
+// workers of +-s_i is formed as (sum of all s_i) - 2 (sum of the s_i whose bit is set): one
+// predicated binary64 add per worker, and exact wherever the plain sum is.
+__global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffers b, float* __restrict__ theta,
+                                                               HyperParams hp,
+                                                               const __grid_constant__ SegParams sp_) {
     __shared__ uint32_t sh_bits[kApplyChunk][32];
     __shared__ double sh_s[kApplyChunk];
-    const TileInfo ti = load_tile(t.tiles, blockIdx.x >> 3);
+    const int tile = blockIdx.x >> 3;
+    const TileInfo ti = sp_.nseg ? find_tile(sp_, tile) : load_tile(t.tiles, tile);
     const int blk = ti.blk;
     const int len = ti.len;
     const int rs = ti.r0 + (int)(blockIdx.x & 7) * kWarpSpan;  // first coordinate of this CTA, relative to the block
     if (rs >= len) return;
     const int r = rs + (int)threadIdx.x * 4;
+    const int64_t o = ti.o;
+    float* gbar = b.gbar + o;
+    float* m = b.m + o;
+    float* v = b.v + o;
+    float* vh = b.vhat + o;
+    float* th = theta + o;
+    const int cls = align_class(m);  // all five vectors are 16-byte aligned at coordinate 0
+    const bool full = r + 3 < len;
+    float4 mm = make_float4(0.f, 0.f, 0.f, 0.f), vv = mm, hh = mm, tt = mm;
+    if (full) {
+        mm = load4(m + r, cls);
+        vv = load4(v + r, cls);
+        hh = load4(vh + r, cls);
+        tt = load4(th + r, cls);
+    }
     const int wsel = threadIdx.x >> 3, nsh = (threadIdx.x & 7) * 4;
-
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    const size_t wbase = (size_t)b.word_off[blk] + (size_t)(rs >> 5);
+    const size_t wbase = (size_t)(sp_.nseg ? (int64_t)sp_.wofs[ti.seg] : b.word_off[blk]) + (size_t)(rs >> 5);
     const int wl = threadIdx.x & 31, wr = threadIdx.x >> 5;  // word and worker this thread stages
     const bool word_live = rs + wl * 32 < len;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0, all = 0.0;
     for (int i0 = 0; i0 < t.n; i0 += kApplyChunk) {
         const int nc = (t.n - i0 < kApplyChunk) ? t.n - i0 : kApplyChunk;
         __syncthreads();
@@ -178,26 +235,22 @@ __global__ void __launch_bounds__(kThreads, 6) bs_apply_kernel(Tables t, BsBuffe
 #pragma unroll 4
         for (int c = 0; c < nc; ++c) {
             const double s = sh_s[c];
-            const double ns = -s;
             const uint32_t nib = sh_bits[c][wsel] >> nsh;
-            a0 += (nib & 1u) ? ns : s;
-            a1 += (nib & 2u) ? ns : s;
-            a2 += (nib & 4u) ? ns : s;
-            a3 += (nib & 8u) ? ns : s;
+            all += s;
+            if (nib & 1u) a0 += s;
+            if (nib & 2u) a1 += s;
+            if (nib & 4u) a2 += s;
+            if (nib & 8u) a3 += s;
         }
     }
+    a0 = all - (a0 + a0);
+    a1 = all - (a1 + a1);
+    a2 = all - (a2 + a2);
+    a3 = all - (a3 + a3);
     if (r >= len) return;
-    const int64_t o = ti.o;
-    float* gbar = b.gbar + o;
-    float* m = b.m + o;
-    float* v = b.v + o;
-    float* vh = b.vhat + o;
-    float* th = theta + o;
-    const int cls = align_class(m);  // all five vectors are 16-byte aligned at coordinate 0
     const float gb[4] = {mean_from_acc(a0, hp.nf), mean_from_acc(a1, hp.nf), mean_from_acc(a2, hp.nf),
                          mean_from_acc(a3, hp.nf)};
-    if (r + 3 < len) {
-        float4 mm = load4(m + r, cls), vv = load4(v + r, cls), hh = load4(vh + r, cls), tt = load4(th + r, cls);
+    if (full) {
         amsgrad_update(gb[0], mm.x, vv.x, hh.x, tt.x, hp);
         amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);
         amsgrad_update(gb[2], mm.z, vv.z, hh.z, tt.z, hp);
@@ -211,13 +264,13 @@ __global__ void __launch_bounds__(kThreads, 6) bs_apply_kernel(Tables t, BsBuffe
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             if (r + k < len) {
-                float mm = m[r + k], vv = v[r + k], hh = vh[r + k], tt = th[r + k];
-                amsgrad_update(gb[k], mm, vv, hh, tt, hp);
+                float m1 = m[r + k], v1 = v[r + k], h1 = vh[r + k], t1 = th[r + k];
+                amsgrad_update(gb[k], m1, v1, h1, t1, hp);
                 gbar[r + k] = gb[k];
-                m[r + k] = mm;
-                v[r + k] = vv;
-                vh[r + k] = hh;
-                th[r + k] = tt;
+                m[r + k] = m1;
+                v[r + k] = v1;
+                vh[r + k] = h1;
+                th[r + k] = t1;
             }
         }
     }
@@ -243,7 +296,7 @@ cudaError_t launch_bs_scales(compams_context* c) {
 cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     BsBuffers b = c->bs;
     b.scales_cur = c->scales[c->scales_cur];
-    bs_apply_kernel<<<(unsigned)c->tab.ntiles * kWarps, kThreads, 0, c->stream>>>(c->tab, b, theta, c->hp);
+    bs_apply_kernel<<<(unsigned)c->tab.ntiles * kWarps, kThreads, 0, c->stream>>>(c->tab, b, theta, c->hp, c->segp);
     return cudaGetLastError();
 }
 

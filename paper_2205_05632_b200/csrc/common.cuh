@@ -45,6 +45,7 @@ struct SegParams {
     int32_t tile0[kParamSegs + 1];  // first tile of each tiled block, then the total
     int32_t len[kParamSegs];
     int32_t blk[kParamSegs];
+    int32_t wofs[kParamSegs];  // Block-Sign: first sign word of the block within a worker's row of words
     int64_t o[kParamSegs];
 };
 

@@ -64,6 +64,7 @@ struct BsBuffers {
     const float* scales_prev; // [n, M]
     float* scales_cur;        // [n, M]
     double* tile_sum;         // [n, ntiles]
+    uint2* edge;              // [n, ntiles] a tile's share of the sign words it has in common with its neighbours
     float *gbar, *m, *v, *vhat;
 };
 
@@ -85,10 +86,10 @@ struct TopkBuffers {
     uint32_t* sel_ticket;      // [n * long lists, 2] slices arrived; threshold-bin candidates appended
     uint2* sel_surv;           // [n * long lists, kSurvCap] threshold-bin candidates of a long list
     double* acc;               // [d] binary64 accumulator, used only by entries that overflow their bucket
-    const uint32_t* kept_prev; // [n, map_words] bit j of row i: coordinate j was kept last step and its e is still
+    const uint32_t* kept_prev; // [map_words] bit i d + j: worker i kept coordinate j last step and its e is still
                                // to be zeroed (null when E is up to date)
-    uint32_t* kept_cur;        // [n, map_words] receives this step's kept coordinates
-    int64_t map_words;         // 32-bit words per worker row of a kept map: ceil(d / 32)
+    uint32_t* kept_cur;        // [map_words] receives this step's kept coordinates
+    int64_t map_words;         // 32-bit words of a kept map: ceil(n d / 32), one bit per element of E
     uint2* bucket;             // [nbucket, bucket_cap] (coordinate inside the bucket, bits of x) per kept entry
     uint32_t* bcount;          // [nbucket] entries appended this step (may exceed bucket_cap)
     uint32_t* bdirty;          // [nbucket] 1: some entries of this bucket went to acc instead

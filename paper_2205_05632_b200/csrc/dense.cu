@@ -84,6 +84,11 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
         vh = *reinterpret_cast<const float4*>(b.vhat + j);
         th = *reinterpret_cast<const float4*>(theta + j);
     }
+    // so is the bucket's first round of entries, before its fill count is known (the slots exist
+    // whatever they hold; an entry is used only if the count covers it)
+    const uint2* ent = b.bucket + (size_t)T * (size_t)b.bucket_cap;
+    uint2 first = make_uint2(0u, 0u);
+    if (threadIdx.x < (uint32_t)b.bucket_cap) first = ent[threadIdx.x];
     const uint32_t appended = b.bcount[T];
     const uint32_t cnt = appended < (uint32_t)b.bucket_cap ? appended : (uint32_t)b.bucket_cap;
     const bool dirty = b.bdirty[T] != 0u;
@@ -92,8 +97,8 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
     sacc[loc + 2] = 0.0;
     sacc[loc + 3] = 0.0;
     __syncthreads();
-    const uint2* ent = b.bucket + (size_t)T * (size_t)b.bucket_cap;
-    for (uint32_t e = threadIdx.x; e < cnt; e += kThreads) {
+    if (threadIdx.x < cnt) atomicAdd(&sacc[first.x], (double)__uint_as_float(first.y));
+    for (uint32_t e = threadIdx.x + kThreads; e < cnt; e += kThreads) {
         const uint2 cv = ent[e];
         atomicAdd(&sacc[cv.x], (double)__uint_as_float(cv.y));
     }

@@ -73,62 +73,57 @@ __device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int len
 // ------------------------------------------------------------------------------------------
 // sweep: x = g + e -> E; keys >= tau_hat go to the candidate list
 
-// Bits j .. j+3 of one worker's kept map (bit j of the row = coordinate j), in the low 4 bits.
-__device__ __forceinline__ uint32_t kept_bits4(const uint32_t* __restrict__ row, int64_t map_words, uint32_t j) {
-    const uint32_t w = j >> 5, sh = j & 31u;
-    uint32_t bits = __ldg(row + w) >> sh;
-    if (sh > 28u && (int64_t)w + 1 < map_words) bits |= __ldg(row + w + 1) << (32u - sh);
-    return bits & 0xfu;
-}
-
+// One tile of the sweep. The tile starts at r0 (relative to the block), which is the block's tile
+// boundary shifted down to a 128-byte line of G and E: r0 may be negative and the tile may reach
+// past the block; such coordinates are skipped. `row0` is the index of the block's first element
+// in E ([n, d] flattened), which is also its bit in the kept map; row0 + r0 is a multiple of 32.
 template <bool FULL>
 __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int r0,
-                                                int warp, int lane, uint32_t tau_hat, uint32_t coord0,
+                                                int warp, int lane, uint32_t tau_hat, uint32_t coord0, int64_t row0,
                                                 uint2* sh_cand, uint32_t* sh_cnt, uint32_t* g_cnt, uint2* g_out,
                                                 uint32_t cap, const uint32_t* __restrict__ kept, int64_t map_words) {
-    const int cg_ = align_class(g), ce = align_class(e);
-    // kept map of this warp's 1024 coordinates: when the block starts on a word boundary, lane l
-    // fetches word l once and the iterations pick their nibbles with shuffles
-    const bool map_fast = kept != nullptr && (coord0 & 31u) == 0u;
+    const int cg_ = align_class(g + r0), ce = align_class(e + r0);
+    // kept map of this warp's 1024 elements: lane l fetches word l once and the iterations pick
+    // their nibbles with shuffles
     uint32_t mapw = 0u;
-    if (map_fast) {
-        const int64_t w = (int64_t)((coord0 + (uint32_t)lane_r(r0, warp, 0, 0)) >> 5) + lane;
+    if (kept != nullptr) {
+        const int64_t w = ((row0 + lane_r(r0, warp, 0, 0)) >> 5) + lane;
         mapw = w < map_words ? __ldg(kept + w) : 0u;
     }
 #pragma unroll
     for (int bt = 0; bt < kIters / 2; ++bt) {
         float4 gv[2], ev[2];
-        uint32_t kb4[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int r = lane_r(r0, warp, bt * 2 + u, lane);
-            if (FULL || r + 3 < len) {
+            if (FULL || (r >= 0 && r + 3 < len)) {
                 gv[u] = load4_stream(g + r, cg_);
                 ev[u] = load4(e + r, ce);
             } else {
                 float gt[4], et[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    gt[k] = (r + k < len) ? __ldg(g + r + k) : 0.0f;
-                    et[k] = (r + k < len) ? e[r + k] : 0.0f;
+                    const bool live = (unsigned)(r + k) < (unsigned)len;
+                    gt[k] = live ? __ldg(g + r + k) : 0.0f;
+                    et[k] = live ? e[r + k] : 0.0f;
                 }
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
                 ev[u] = make_float4(et[0], et[1], et[2], et[3]);
             }
-            // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, line 8)
-            kb4[u] = (kept && !map_fast) ? kept_bits4(kept, map_words, coord0 + (uint32_t)r) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int r = lane_r(r0, warp, bt * 2 + u, lane);
-            if (map_fast)  // after the batch's loads have been issued: the shuffle waits for the map word
-                kb4[u] = (__shfl_sync(0xffffffffu, mapw, (bt * 2 + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
+            // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, line 8).
+            // Placed after the batch's loads have been issued: the shuffle waits for the map word.
+            const uint32_t kb4 =
+                (__shfl_sync(0xffffffffu, mapw, (bt * 2 + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
             float xs[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float ek = ((kb4[u] >> k) & 1u) ? 0.0f : lane_elem(ev[u], k);
+                const float ek = ((kb4 >> k) & 1u) ? 0.0f : lane_elem(ev[u], k);
                 xs[k] = __fadd_rn(lane_elem(gv[u], k), ek);  // line 7: x = g + e
-                if ((FULL || r + k < len) && mag_key(xs[k]) >= tau_hat) {
+                if ((FULL || (unsigned)(r + k) < (unsigned)len) && mag_key(xs[k]) >= tau_hat) {
                     const uint2 cv = make_uint2(coord0 + (uint32_t)(r + k), __float_as_uint(xs[k]));
                     const uint32_t slot = atomicAdd(sh_cnt, 1u);
                     if (slot < (uint32_t)kTileCand) {
@@ -139,17 +134,20 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
                     }
                 }
             }
-            if (FULL || r + 3 < len) {
+            if (FULL || (r >= 0 && r + 3 < len)) {
                 store4(e + r, ce, make_float4(xs[0], xs[1], xs[2], xs[3]));
             } else {
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    if (r + k < len) e[r + k] = xs[k];
+                    if ((unsigned)(r + k) < (unsigned)len) e[r + k] = xs[k];
             }
         }
     }
 }
 
+// Tiles are shifted down by (i d + o) mod 32, the position of the block's first element within a
+// 128-byte line of G and E, so that every warp access covers whole lines (with rows that start
+// mid-line a warp's 512 bytes straddle five lines instead of four: measured 7 % slower).
 __global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const float* __restrict__ G,
                                                                  const __grid_constant__ SegParams sp_) {
     __shared__ uint2 sh_cand[kTileCand];
@@ -165,15 +163,16 @@ __global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkB
     uint2* out = b.cand + (size_t)i * (size_t)b.cand_total + (size_t)si->cand_off;
     if (threadIdx.x == 0) sh_cnt = 0u;
     __syncthreads();
-    const float* g = G + (size_t)i * (size_t)t.d + (size_t)ti.o;
-    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
-    const uint32_t* kept = b.kept_prev ? b.kept_prev + (size_t)i * (size_t)b.map_words : nullptr;
-    if (ti.r0 + kTile <= ti.len)
-        topk_sweep_tile<true>(g, e, ti.len, ti.r0, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
-                              &st->cand_count, out, cap, kept, b.map_words);
+    const int64_t row0 = (int64_t)i * t.d + ti.o;
+    const float* g = G + row0;
+    float* e = b.E + row0;
+    const int r0s = ti.r0 - (int)(row0 & 31);
+    if (r0s >= 0 && r0s + kTile <= ti.len)
+        topk_sweep_tile<true>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, row0, sh_cand, &sh_cnt,
+                              &st->cand_count, out, cap, b.kept_prev, b.map_words);
     else
-        topk_sweep_tile<false>(g, e, ti.len, ti.r0, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
-                               &st->cand_count, out, cap, kept, b.map_words);
+        topk_sweep_tile<false>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, row0, sh_cand, &sh_cnt,
+                               &st->cand_count, out, cap, b.kept_prev, b.map_words);
     __syncthreads();
     const uint32_t cnt = sh_cnt;
     if (cnt == 0u) return;
@@ -1129,33 +1128,26 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
         b.bdirty[T] = 1u;
     }
     // the coordinate's e becomes 0 (line 8: e = x - x): recorded in the kept map, applied when E is next read
-    const int64_t i = p / b.K;
-    atomicOr(b.kept_cur + (size_t)i * (size_t)b.map_words + ((uint32_t)j >> 5), 1u << ((uint32_t)j & 31u));
+    const int64_t f = (p / b.K) * t.d + j;  // the element's index in E, [n, d] flattened
+    atomicOr(b.kept_cur + (size_t)(f >> 5), 1u << (uint32_t)(f & 31));
 }
 
 // E holds x at the coordinates kept in the last step: zero them (Algorithm 2, line 8), one thread per word.
-__global__ void __launch_bounds__(kThreads) topk_materialize_kernel(int32_t n, int64_t d, int64_t map_words,
+__global__ void __launch_bounds__(kThreads) topk_materialize_kernel(int64_t nd, int64_t map_words,
                                                                     const uint32_t* __restrict__ kept,
                                                                     float* __restrict__ E) {
     const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= (int64_t)n * map_words) return;
+    if (q >= map_words) return;
     uint32_t w = kept[q];
-    const int64_t i = q / map_words;
-    float* e = E + (size_t)i * (size_t)d + (size_t)(q % map_words) * 32;
+    float* e = E + (size_t)q * 32;
     while (w) {
         const int k = __ffs(w) - 1;
         w &= w - 1;
-        e[k] = 0.0f;
+        if (q * 32 + k < nd) e[k] = 0.0f;
     }
 }
 
 // ------------------------------------------------------------------------------------------
-
-static int persistent_grid(const compams_context* c, int64_t items, int ctas_per_sm) {
-    int64_t cap = (int64_t)c->num_sms * ctas_per_sm;
-    if (items < 1) items = 1;
-    return (int)(items < cap ? items : cap);
-}
 
 cudaError_t launch_topk_small(compams_context* c, const float* grads) {
     dim3 grid((unsigned)c->tk.nsmall, (unsigned)c->n);
@@ -1199,9 +1191,9 @@ cudaError_t launch_topk_dense(compams_context* c) {
 }
 
 cudaError_t launch_topk_materialize(compams_context* c) {
-    const int64_t words = (int64_t)c->n * c->tk.map_words;
+    const int64_t words = c->tk.map_words;
     topk_materialize_kernel<<<(unsigned)((words + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
-        c->n, c->d, c->tk.map_words, c->keptmap[c->map_cur], c->E);
+        (int64_t)c->n * c->d, c->tk.map_words, c->keptmap[c->map_cur], c->E);
     return cudaGetLastError();
 }
 

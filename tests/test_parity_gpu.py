@@ -59,6 +59,33 @@ def test_rows_not_multiple_of_four_use_all_alignment_classes():
     _pair_run(4, d, [0, d], TOPK, 1.0, _randn(4, d), steps=3)
 
 
+@pytest.mark.parametrize("shift", [1, 2, 3])
+def test_gradient_buffer_off_the_16_byte_grid(shift):
+    # the caller's G may start anywhere on the 4-byte grid, while E is the library's own: the two no
+    # longer share their alignment and G is read with narrower loads; results must not change
+    n, d = 3, 2 * 8192 + 4101
+    offs = [0, 4099, d]
+    for comp, ratio in ((TOPK, 0.05), (BLOCKSIGN, 1.0), (TOPK, 1.0)):
+        a = CompAMS(n, d, offs, comp, ratio)
+        b = CompAMS(n, d, offs, comp, ratio)
+        ta = torch.zeros(d, device="cuda")
+        tb = torch.zeros(d, device="cuda")
+        gen = torch.Generator(device="cuda").manual_seed(77)
+        for t in range(3):
+            G = torch.randn(n, d, generator=gen, device="cuda")
+            store = torch.empty(n * d + 8, device="cuda")
+            Gs = store[shift:shift + n * d].view(n, d)
+            Gs.copy_(G)
+            assert Gs.data_ptr() % 16 == 4 * shift
+            a.step(G, ta)
+            b.step(Gs, tb)
+        for name in ("E", "m", "v", "vhat", "gbar"):
+            assert torch.equal(a.buffer(name).view(torch.int32), b.buffer(name).view(torch.int32)), name
+        assert torch.equal(ta.view(torch.int32), tb.view(torch.int32))
+        a.close()
+        b.close()
+
+
 def test_blocks_of_size_one_and_tiny():
     d = 200
     offs = list(range(0, 101)) + [110, 150, 200]
