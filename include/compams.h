@@ -162,6 +162,39 @@ int compams_set_stream(compams_handle h, void* cuda_stream);
 int compams_set_lr(compams_handle h, float lr);
 
 /*
+ * compams_get_state / compams_set_state - checkpoint and restore what Algorithm 2 carries from one
+ * iteration to the next: the workers' error accumulators e_{t,i} (line 8) and the server's m_t, v_t,
+ * v-hat_t (lines 13-15). theta is the caller's own tensor and the step counter does not enter the
+ * update (Algorithm 1 has no bias correction), so these four are the whole state.
+ *
+ *   e         DEVICE, [n, d] packed rows, or null to skip. With k_b = d_b in every block the
+ *             accumulators are identically zero and not stored: get writes zeros, set ignores e.
+ *   m, v, vhat  DEVICE, [d] each, or null to skip.
+ *
+ * get copies out the values line 8 defines (a residual still to be finished is finished first);
+ * set copies in and forgets what the library had derived from earlier steps (threshold
+ * predictions), which changes the path a selection takes, never its result. Both run on the
+ * handle's stream, asynchronously; the caller's buffers must stay valid until that work is done.
+ * A run continued from a restored state is bit-identical to the uninterrupted one.
+ */
+int compams_get_state(compams_handle h, float* e, float* m, float* v, float* vhat);
+int compams_set_state(compams_handle h, const float* e, const float* m, const float* v, const float* vhat);
+
+/*
+ * compams_bits_transmitted - worker-to-server traffic of all steps so far, in bits, under the
+ * accounting of Section 5.2 ("Communication Efficiency": 32 bits per floating-point number).
+ *
+ *   out   host, uint64[3]:
+ *         [0] what full-precision gradients would have cost: 32 n d per step;
+ *         [1] the compressed payload: per worker and step 32 bits per kept value (Top-k), or one
+ *             bit per coordinate plus 32 bits per block scale (Block-Sign); equal to [0] when
+ *             every block keeps all its coordinates;
+ *         [2] the 32-bit coordinate indices that accompany Top-k values (0 otherwise). The
+ *             paper's "around 100x" for Top-0.01 is [0] / [1]; a wire format also pays [2].
+ */
+int compams_bits_transmitted(compams_handle h, uint64_t* out);
+
+/*
  * compams_get_buffer - device pointer and element count of one of the handle's buffers.
  *
  *   which     a compams_buffer value.

@@ -74,6 +74,12 @@ def load_library() -> ctypes.CDLL:
     L.compams_set_stream.argtypes = [H, c.c_void_p]
     L.compams_set_lr.restype = c.c_int
     L.compams_set_lr.argtypes = [H, c.c_float]
+    L.compams_get_state.restype = c.c_int
+    L.compams_get_state.argtypes = [H, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    L.compams_set_state.restype = c.c_int
+    L.compams_set_state.argtypes = [H, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    L.compams_bits_transmitted.restype = c.c_int
+    L.compams_bits_transmitted.argtypes = [H, c.POINTER(c.c_uint64)]
     L.compams_get_buffer.restype = c.c_int
     L.compams_get_buffer.argtypes = [H, c.c_int32, c.POINTER(c.c_void_p), c.POINTER(c.c_int64)]
     L.compams_check_status.restype = c.c_int
@@ -176,6 +182,35 @@ class CompAMS:
 
     def set_lr(self, lr: float) -> None:
         _check(self._L.compams_set_lr(self._h, float(lr)), "compams_set_lr")
+
+    def get_state(self) -> dict:
+        """The state Algorithm 2 carries between iterations, as new CUDA tensors: e [n, d]; m, v, vhat [d]."""
+        dev = torch.device("cuda", torch.cuda.current_device())
+        out = {"e": torch.empty(self.n, self.d, dtype=torch.float32, device=dev)}
+        for name in ("m", "v", "vhat"):
+            out[name] = torch.empty(self.d, dtype=torch.float32, device=dev)
+        _check(self._L.compams_get_state(self._h, *(ctypes.c_void_p(out[k].data_ptr()) for k in ("e", "m", "v", "vhat"))),
+               "compams_get_state")
+        return out
+
+    def set_state(self, state: dict) -> None:
+        """Restore (part of) a state returned by get_state(); missing keys are left as they are."""
+        ptrs = []
+        for name, shape in (("e", (self.n, self.d)), ("m", (self.d,)), ("v", (self.d,)), ("vhat", (self.d,))):
+            t = state.get(name)
+            if t is None:
+                ptrs.append(ctypes.c_void_p(0))
+                continue
+            if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == shape):
+                raise CompAMSError("state[%r] must be a contiguous float32 CUDA tensor of shape %r" % (name, shape))
+            ptrs.append(ctypes.c_void_p(t.data_ptr()))
+        _check(self._L.compams_set_state(self._h, *ptrs), "compams_set_state")
+
+    def bits_transmitted(self) -> dict:
+        """Worker-to-server bits so far under the accounting of Section 5.2 (32 bits per float)."""
+        out = (ctypes.c_uint64 * 3)()
+        _check(self._L.compams_bits_transmitted(self._h, out), "compams_bits_transmitted")
+        return {"full_precision": int(out[0]), "payload": int(out[1]), "topk_indices": int(out[2])}
 
     def step(self, grads: torch.Tensor, theta: torch.Tensor) -> None:
         if not (grads.is_cuda and theta.is_cuda):

@@ -222,6 +222,8 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
             for (size_t k = 0; k < seg0.size(); ++k)
                 seg0[k].fallback = c->seg_cap_host[k % (size_t)c->tab.nseg] ? 0u : 1u;
             RC(dev_upload(c, &t.seg, seg0));
+            c->seg_init_host = seg0;
+            c->dense_count_init = never * (uint32_t)n;
             std::vector<uint32_t> dc(1, never * (uint32_t)n);
             RC(dev_upload(c, &t.dense_count, dc));
         }
@@ -314,6 +316,7 @@ int run_kernel(compams_context* c, int kernel, F&& launch) {
 }
 
 int step_device(compams_context* c, const float* grads, float* theta) {
+    ++c->steps_done;
     if (c->compressor == COMPAMS_TOPK && c->identity) {
         return run_kernel(c, COMPAMS_K_DENSE_MEAN_AMSGRAD, [&] { return launch_dense_mean_amsgrad(c, grads, theta); });
     }
@@ -449,6 +452,75 @@ int compams_set_lr(compams_handle c, float lr) {
     return COMPAMS_OK;
 }
 
+// Finishes line 8 where it has been deferred, so that E holds e.
+static int finish_residual(compams_context* c) {
+    if (c->compressor == COMPAMS_TOPK && !c->identity && c->e_mask_pending) {
+        RC(run_kernel(c, COMPAMS_K_TOPK_MATERIALIZE, [&] { return launch_topk_materialize(c); }));
+        c->e_mask_pending = false;
+    }
+    if (c->compressor == COMPAMS_BLOCKSIGN && c->e_is_x) {
+        RC(run_kernel(c, COMPAMS_K_BS_MATERIALIZE, [&] { return launch_bs_materialize(c); }));
+        c->e_is_x = false;
+    }
+    return COMPAMS_OK;
+}
+
+int compams_get_state(compams_handle c, float* e, float* m, float* v, float* vhat) {
+    if (!c) return COMPAMS_ERR_INVALID_ARG;
+    CU(cudaSetDevice(c->device));
+    const size_t nd = (size_t)c->n * (size_t)c->d * sizeof(float), db = (size_t)c->d * sizeof(float);
+    if (e) {
+        if (c->E) {
+            RC(finish_residual(c));
+            CU(cudaMemcpyAsync(e, c->E, nd, cudaMemcpyDeviceToDevice, c->stream));
+        } else {
+            CU(cudaMemsetAsync(e, 0, nd, c->stream));
+        }
+    }
+    if (m) CU(cudaMemcpyAsync(m, c->m, db, cudaMemcpyDeviceToDevice, c->stream));
+    if (v) CU(cudaMemcpyAsync(v, c->v, db, cudaMemcpyDeviceToDevice, c->stream));
+    if (vhat) CU(cudaMemcpyAsync(vhat, c->vhat, db, cudaMemcpyDeviceToDevice, c->stream));
+    return COMPAMS_OK;
+}
+
+int compams_set_state(compams_handle c, const float* e, const float* m, const float* v, const float* vhat) {
+    if (!c) return COMPAMS_ERR_INVALID_ARG;
+    CU(cudaSetDevice(c->device));
+    const size_t nd = (size_t)c->n * (size_t)c->d * sizeof(float), db = (size_t)c->d * sizeof(float);
+    if (e && c->E) {
+        CU(cudaMemcpyAsync(c->E, e, nd, cudaMemcpyDeviceToDevice, c->stream));
+        // E now holds e itself; predictions made from the replaced accumulators are dropped
+        c->e_is_x = false;
+        c->e_mask_pending = false;
+        if (c->tk.seg && !c->seg_init_host.empty()) {
+            CU(cudaMemcpyAsync(c->tk.seg, c->seg_init_host.data(), c->seg_init_host.size() * sizeof(SegState),
+                               cudaMemcpyHostToDevice, c->stream));
+            CU(cudaMemcpyAsync(c->tk.dense_count, &c->dense_count_init, sizeof(uint32_t), cudaMemcpyHostToDevice,
+                               c->stream));
+        }
+    }
+    if (m) CU(cudaMemcpyAsync(c->m, m, db, cudaMemcpyDeviceToDevice, c->stream));
+    if (v) CU(cudaMemcpyAsync(c->v, v, db, cudaMemcpyDeviceToDevice, c->stream));
+    if (vhat) CU(cudaMemcpyAsync(c->vhat, vhat, db, cudaMemcpyDeviceToDevice, c->stream));
+    return COMPAMS_OK;
+}
+
+int compams_bits_transmitted(compams_handle c, uint64_t* out) {
+    if (!c || !out) return COMPAMS_ERR_INVALID_ARG;
+    const uint64_t full = 32ull * (uint64_t)c->n * (uint64_t)c->d;
+    uint64_t payload = full, index = 0;
+    if (c->compressor == COMPAMS_BLOCKSIGN) {
+        payload = (uint64_t)c->n * ((uint64_t)c->d + 32ull * (uint64_t)c->M);
+    } else if (!c->identity) {
+        payload = 32ull * (uint64_t)c->n * (uint64_t)c->K;
+        index = payload;
+    }
+    out[0] = full * c->steps_done;
+    out[1] = payload * c->steps_done;
+    out[2] = index * c->steps_done;
+    return COMPAMS_OK;
+}
+
 int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t* count) {
     if (!c || !dev_ptr || !count) return COMPAMS_ERR_INVALID_ARG;
     void* p = nullptr;
@@ -457,14 +529,7 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
     const bool sign = c->compressor == COMPAMS_BLOCKSIGN;
     switch (which) {
         case COMPAMS_BUF_E:
-            if (topk && c->e_mask_pending) {
-                RC(run_kernel(c, COMPAMS_K_TOPK_MATERIALIZE, [&] { return launch_topk_materialize(c); }));
-                c->e_mask_pending = false;
-            }
-            if (sign && c->e_is_x) {
-                RC(run_kernel(c, COMPAMS_K_BS_MATERIALIZE, [&] { return launch_bs_materialize(c); }));
-                c->e_is_x = false;
-            }
+            RC(finish_residual(c));
             p = c->E;
             cnt = (int64_t)c->n * c->d;
             break;

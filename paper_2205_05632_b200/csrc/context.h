@@ -127,6 +127,9 @@ struct compams_context {
     int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists a cluster selects from
     int n_sel_small = 0, n_sel_big = 0;
     int sel_parts = 1;  // slices a long candidate list is cut into
+    std::vector<compams::SegState> seg_init_host;  // Top-k: the segments' state before the first step (set_state restores it)
+    uint32_t dense_count_init = 0;
+    uint64_t steps_done = 0;
     uint32_t* keptmap[2] = {nullptr, nullptr};  // Top-k: kept maps of this and the previous step
     int map_cur = 0;
     bool e_mask_pending = false;  // Top-k: E still holds x at the coordinates kept in the last step

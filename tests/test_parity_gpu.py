@@ -293,3 +293,79 @@ def test_set_lr_takes_effect_on_the_next_step():
     opt.step(G, theta)
     assert torch.equal(theta, moved)
     opt.close()
+
+
+# ------------------------------------------------------------------ checkpoint / restore, traffic accounting
+
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.02), (BLOCKSIGN, 1.0), (TOPK, 1.0)])
+def test_restored_state_continues_bit_identically(comp, ratio):
+    n, d = 3, 5 * 8192 + 1234
+    offs = [0, 3000, 20000, d]
+    gen = torch.Generator(device="cuda").manual_seed(9)
+    G = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(6)]
+    a = CompAMS(n, d, offs, comp, ratio)
+    theta_a = torch.zeros(d, device="cuda")
+    for g in G[:3]:
+        a.step(g, theta_a)
+    saved = {k: v.clone() for k, v in a.get_state().items()}
+    theta_saved = theta_a.clone()
+    for g in G[3:]:
+        a.step(g, theta_a)
+    # the saved e is what line 8 defines, not the library's deferred form of it
+    b = CompAMS(n, d, offs, comp, ratio)
+    b.set_state(saved)
+    if not (comp == TOPK and ratio == 1.0):
+        assert torch.equal(b.buffer("E"), saved["e"])
+    else:
+        assert not saved["e"].any()
+    theta_b = theta_saved.clone()
+    for g in G[3:]:
+        b.step(g, theta_b)
+    assert torch.equal(theta_a.view(torch.int32), theta_b.view(torch.int32))
+    sa, sb = a.get_state(), b.get_state()
+    for k in sa:
+        assert torch.equal(sa[k].view(torch.int32), sb[k].view(torch.int32)), k
+    assert a.check_status() == 0 and b.check_status() == 0
+    a.close()
+    b.close()
+
+
+def test_get_state_matches_the_oracle_and_leaves_the_run_unchanged():
+    from parity import Pair, close
+    n, d = 2, 3 * 8192 + 17
+    for comp, ratio in ((TOPK, 0.01), (BLOCKSIGN, 1.0)):
+        gen = torch.Generator(device="cuda").manual_seed(3)
+        p = Pair(n, d, [0, 5000, d], comp, ratio)
+        try:
+            p.start(torch.zeros(d, device="cuda"))
+            for t in range(4):
+                p.step(torch.randn(n, d, generator=gen, device="cuda"), check_e=False)
+                st = p.gpu.get_state()   # every step: reading the state must not disturb the next one
+                close(st["e"], p.cpu.buffer("E"), "e from get_state", t + 1)
+                close(st["m"], p.cpu.buffer("m"), "m from get_state", t + 1)
+                close(st["vhat"], p.cpu.buffer("vhat"), "vhat from get_state", t + 1)
+        finally:
+            p.close()
+
+
+def test_bits_transmitted_follow_the_32_bit_accounting():
+    n, d = 4, 100000
+    offs = [0, 30000, d]
+    g = torch.zeros(n, d, device="cuda")
+    theta = torch.zeros(d, device="cuda")
+    t = CompAMS(n, d, offs, TOPK, 0.01)
+    for _ in range(3):
+        t.step(g, theta)
+    k = 300 + 700
+    assert t.bits_transmitted() == {"full_precision": 3 * 32 * n * d, "payload": 3 * 32 * n * k,
+                                    "topk_indices": 3 * 32 * n * k}
+    t.close()
+    s = CompAMS(n, d, offs, BLOCKSIGN)
+    s.step(g, theta)
+    s.step(g, theta)
+    assert s.bits_transmitted() == {"full_precision": 2 * 32 * n * d, "payload": 2 * n * (d + 32 * 2), "topk_indices": 0}
+    s.close()
+    f = CompAMS(n, d, offs, TOPK, 1.0)
+    f.step(g, theta)
+    assert f.bits_transmitted() == {"full_precision": 32 * n * d, "payload": 32 * n * d, "topk_indices": 0}
+    f.close()
