@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffe
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     __shared__ uint32_t sh_first[kWarps];
+    allow_dependents();
     const int tile = blockIdx.x;
     const int i = blockIdx.y;
     const TileInfo ti = sp_.nseg ? find_tile(sp_, tile) : load_tile(t.tiles, tile);
@@ -148,6 +149,8 @@ __global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffe
 // One CTA per (worker, block): scale = ||x_B||_1 / d_B from the tile sums (Definition 2).
 __global__ void __launch_bounds__(kThreads) bs_scales_kernel(Tables t, BsBuffers b) {
     __shared__ double red[kWarps];
+    allow_dependents();
+    dependency_wait();  // the sweep's tile sums and word shares
     const int blk = blockIdx.x, i = blockIdx.y;
     const SegInfo* si = t.segs + blk;
     const double* ts = b.tile_sum + (size_t)i * t.ntiles + si->tile0;
@@ -220,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
         hh = load4(vh + r, cls);
         tt = load4(th + r, cls);
     }
+    dependency_wait();  // the state above was last written a step ago; sign words and scales are this step's
     const int wsel = threadIdx.x >> 3, nsh = (threadIdx.x & 7) * 4;
     const size_t wbase = (size_t)(sp_.nseg ? (int64_t)sp_.wofs[ti.seg] : b.word_off[blk]) + (size_t)(rs >> 5);
     const int wl = threadIdx.x & 31, wr = threadIdx.x >> 5;  // word and worker this thread stages
@@ -289,15 +293,14 @@ cudaError_t launch_bs_scales(compams_context* c) {
     dim3 grid((unsigned)c->M, (unsigned)c->n);
     BsBuffers b = c->bs;
     b.scales_cur = c->scales[c->scales_cur];
-    bs_scales_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b);
-    return cudaGetLastError();
+    return launch_after(bs_scales_kernel, grid, dim3(kThreads), c->stream, c->tab, b);
 }
 
 cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     BsBuffers b = c->bs;
     b.scales_cur = c->scales[c->scales_cur];
-    bs_apply_kernel<<<(unsigned)c->tab.ntiles * kWarps, kThreads, 0, c->stream>>>(c->tab, b, theta, c->hp, c->segp);
-    return cudaGetLastError();
+    return launch_after(bs_apply_kernel, dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), c->stream, c->tab, b,
+                        theta, c->hp, c->segp);
 }
 
 cudaError_t launch_bs_materialize(compams_context* c) {

@@ -158,6 +158,30 @@ __device__ __forceinline__ TileInfo find_tile(const SegParams& sp, int tile) {
     return ti;
 }
 
+// Programmatic dependent launch: a kernel launched with launch_after() may start while the kernel
+// before it on the stream is still draining. It may touch nothing that kernel (or any earlier one it
+// has not been ordered after) writes until dependency_wait() has returned; what it reads before that
+// - here: optimizer state that only the previous step wrote - overlaps the predecessor's tail.
+// allow_dependents() in the predecessor lets the successor's CTAs in as soon as all of its own have
+// started. Both are no-ops in a plainly launched kernel.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Inclusive scan of one unsigned value per thread across a CTA of kThreads threads.
 // `scratch` holds NWARPS words (the CTA has NWARPS warps). Returns the inclusive prefix; *total receives the CTA sum.
 template <int NWARPS = kWarps>

@@ -84,8 +84,9 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
         vh = *reinterpret_cast<const float4*>(b.vhat + j);
         th = *reinterpret_cast<const float4*>(theta + j);
     }
-    // so is the bucket's first round of entries, before its fill count is known (the slots exist
-    // whatever they hold; an entry is used only if the count covers it)
+    dependency_wait();  // everything below is this step's: the scatter kernel's buckets
+    // the bucket's first round of entries is requested before its fill count is known (the slots
+    // exist whatever they hold; an entry is used only if the count covers it)
     const uint2* ent = b.bucket + (size_t)T * (size_t)b.bucket_cap;
     uint2 first = make_uint2(0u, 0u);
     if (threadIdx.x < (uint32_t)b.bucket_cap) first = ent[threadIdx.x];
@@ -157,8 +158,8 @@ cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, fl
 }
 
 cudaError_t launch_amsgrad(compams_context* c, float* theta) {
-    amsgrad_bucket_kernel<<<(unsigned)c->tk.nbucket, kThreads, 0, c->stream>>>(c->d, c->tk, theta, c->hp);
-    return cudaGetLastError();
+    return launch_after(amsgrad_bucket_kernel, dim3((unsigned)c->tk.nbucket), dim3(kThreads), c->stream, c->d, c->tk, theta,
+                        c->hp);
 }
 
 }  // namespace compams

@@ -1087,6 +1087,7 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 // The same walk zeroes e at the kept coordinates (they were left holding x by the sweep).
 
 __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count) {
+    allow_dependents();
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     // the first n * nseg threads also close the step for one large-block segment each: exactly k_b
     // entries must have been emitted; counters go back to their resting values
