@@ -155,7 +155,7 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
             c->sel_parts = (int)(parts < 1 ? 1 : parts > 64 ? 64 : parts);
             RC(dev_alloc(c, &c->tk.sel_hist, (size_t)lists * kSelBins));
             RC(dev_alloc(c, &c->tk.sel_ticket, (size_t)lists * 2));
-            RC(dev_alloc(c, &c->tk.sel_surv, (size_t)lists * kSurvCap, false));
+            RC(dev_alloc(c, &c->tk.sel_surv, (size_t)lists * kSurvCapBig, false));
         }
     }
     return COMPAMS_OK;

@@ -20,6 +20,7 @@ constexpr int kMaxTimed = 4096;    // event pairs kept for per-kernel timing
 constexpr uint32_t kNoPrediction = 0xffffffffu;  // tau_hat value that no key reaches
 constexpr int kTileCand = 1024;          // candidates one tile can stage in shared memory
 constexpr int kSurvCap = 1536;           // threshold-bin candidates a select can rank in shared memory
+constexpr int kSurvCapBig = 65536;       // threshold-bin candidates of a long list (kept in global memory)
 constexpr int kSelBins = 4096;           // bins of the candidate select's first histogram
 constexpr int kSelectSingleMax = 24576;  // candidate capacity up to which one CTA handles a segment
 
@@ -84,7 +85,7 @@ struct TopkBuffers {
     uint32_t* dense_count;     // [1] segments currently marked for the dense passes
     uint32_t* sel_hist;        // [n * long lists, kSelBins] histogram a long list's slices add into
     uint32_t* sel_ticket;      // [n * long lists, 2] slices arrived; threshold-bin candidates appended
-    uint2* sel_surv;           // [n * long lists, kSurvCap] threshold-bin candidates of a long list
+    uint2* sel_surv;           // [n * long lists, kSurvCapBig] threshold-bin candidates of a long list
     double* acc;               // [d] binary64 accumulator, used only by entries that overflow their bucket
     const uint32_t* kept_prev; // [map_words] bit i d + j: worker i kept coordinate j last step and its e is still
                                // to be zeroed (null when E is up to date)

@@ -586,7 +586,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
     const uint32_t lo = (uint32_t)part * per < c ? (uint32_t)part * per : c;
     const uint32_t hi = (lo + per < c) ? lo + per : c;
     const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
-    uint2* gsurv = b.sel_surv + item * kSurvCap;
+    uint2* gsurv = b.sel_surv + item * kSurvCapBig;
     uint32_t* gscnt = b.sel_ticket + 2 * item + 1;  // survivors appended so far (second word of the pair)
 
     // first pass over the slice (from L2): how many winners, so that they get one contiguous slot range
@@ -627,7 +627,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
             }
             if (__any_sync(0xffffffffu, keep)) {  // rare: only the threshold bin's candidates
                 const uint32_t spos = warp_slot(keep, gscnt, lane);
-                if (keep && spos < (uint32_t)kSurvCap) gsurv[spos] = cv;
+                if (keep && spos < (uint32_t)kSurvCapBig) gsurv[spos] = cv;
             }
         }
     }
@@ -645,7 +645,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
         b.sel_ticket[2 * item + 1] = 0u;
         st->sel_ready = 0u;
     }
-    if (nsurv > (uint32_t)kSurvCap) {
+    if (nsurv > (uint32_t)kSurvCapBig) {
         // too many candidates share the threshold bin (heavily duplicated values): dense passes
         if (threadIdx.x == 0) {
             st->fallback = 1u;
@@ -656,7 +656,71 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
     }
     const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
     uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
-    if (!take_all0) {
+    if (!take_all0 && nsurv > (uint32_t)kSurvCap) {
+        // A very long list leaves more of the threshold bin than shared memory can rank pair by pair.
+        // The survivors differ in the low S key bits and the index; the k_rem-th largest of these
+        // (low bits, lower index first) composites is found digit by digit, 8 bits at a time from
+        // the top, with a 256-bin histogram over the survivors that match the digits found so far.
+        uint32_t* hist = reinterpret_cast<uint32_t*>(surv);  // 256 words of the (here unused) ranking buffer
+        const uint32_t lowmask = S ? ((1u << S) - 1u) : 0u;
+        auto comp_of = [&](const uint2& cv) -> unsigned long long {
+            const uint32_t o = (cv.y & 0x7fffffffu) - tau_hat;
+            return ((unsigned long long)(o & lowmask) << 32) | (unsigned long long)(0xffffffffu - cv.x);
+        };
+        unsigned long long prefix = 0ull;  // digits found so far, right-aligned
+        uint32_t need = k_rem;             // rank still to be located among the survivors matching `prefix`
+        const int top = ((S + 32 + 7) / 8 - 1) * 8;
+        for (int shift = top; shift >= 0; shift -= 8) {
+            __syncthreads();
+            hist[threadIdx.x] = 0u;
+            __syncthreads();
+            for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
+                const unsigned long long cq = comp_of(__ldcg(gsurv + q));
+                const bool match = (shift + 8 >= 64) || ((cq >> (shift + 8)) == prefix);
+                if (match) atomicAdd(&hist[(uint32_t)(cq >> shift) & 255u], 1u);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                uint32_t above = 0;
+                int dsel = 255;
+                for (; dsel > 0; --dsel) {
+                    if (above + hist[dsel] >= need) break;
+                    above += hist[dsel];
+                }
+                sh_base = (uint32_t)dsel;
+                sh_wcnt = above;
+            }
+            __syncthreads();
+            prefix = (prefix << 8) | (unsigned long long)sh_base;
+            need -= sh_wcnt;
+        }
+        // `prefix` is now the composite of the k_rem-th largest survivor (composites are distinct)
+        const unsigned long long thr = prefix;
+        tau = tau_hat + (uint32_t)(((unsigned long long)b0 << S) | (thr >> 32));
+        for (uint32_t q0 = 0; q0 < nsurv; q0 += kThreads) {  // uniform trip count: the loop holds barriers
+            const uint32_t q = q0 + threadIdx.x;
+            uint2 cv = make_uint2(0u, 0u);
+            bool kept = false;
+            if (q < nsurv) {
+                cv = __ldcg(gsurv + q);
+                kept = comp_of(cv) >= thr;
+            }
+            uint32_t tot3;
+            const uint32_t incl = block_inclusive_scan(kept ? 1u : 0u, scratch, &tot3);
+            if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
+            __syncthreads();
+            if (kept) {
+                const uint32_t pos = sh_base + incl - 1u;
+                if (pos < kb) {
+                    b.idx[slot0 + pos] = (int32_t)cv.x;
+                    b.val[slot0 + pos] = __uint_as_float(cv.y);
+                } else {
+                    atomicOr(b.status, 1u);
+                }
+            }
+            __syncthreads();
+        }
+    } else if (!take_all0) {
         for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) surv[q] = __ldcg(gsurv + q);
         __syncthreads();
         // survivor q is kept when fewer than k_rem survivors beat it in (key, lower index first) order

@@ -15,18 +15,29 @@ from paper_2205_05632_b200 import BLOCKSIGN, TOPK, CompAMS
 ATOL, RTOL = 1e-7, 1e-6
 
 
+_CHUNK = 1 << 28  # elements compared at a time: bounds the temporaries at the largest sizes
+
+
 def close(gpu: torch.Tensor, cpu: np.ndarray, what: str, step: int) -> int:
     """Asserts the tolerance elementwise (on the GPU, the arrays can be large). Returns the number of
     elements that are not bit-identical, for reporting."""
-    ref = torch.from_numpy(np.ascontiguousarray(cpu)).to(gpu.device)
-    assert ref.shape == gpu.shape, (what, ref.shape, gpu.shape)
-    bad = (gpu - ref).abs() > (ATOL + RTOL * ref.abs())
-    nbad = int(bad.sum())
-    if nbad:
-        j = int(torch.nonzero(bad.flatten())[0])
-        raise AssertionError("step %d: %s differs at %d element(s); first at flat index %d: gpu=%r cpu=%r" % (
-            step, what, nbad, j, float(gpu.flatten()[j]), float(ref.flatten()[j])))
-    return int((gpu.view(torch.int32) != ref.view(torch.int32)).sum())
+    cpu = np.ascontiguousarray(cpu)
+    assert tuple(cpu.shape) == tuple(gpu.shape), (what, cpu.shape, tuple(gpu.shape))
+    g_flat, c_flat = gpu.reshape(-1), cpu.reshape(-1)
+    inexact = 0
+    for lo in range(0, g_flat.numel(), _CHUNK):
+        hi = min(lo + _CHUNK, g_flat.numel())
+        g = g_flat[lo:hi]
+        ref = torch.from_numpy(c_flat[lo:hi]).to(gpu.device)
+        bad = (g - ref).abs() > (ATOL + RTOL * ref.abs())
+        nbad = int(bad.sum())
+        if nbad:
+            j = int(torch.nonzero(bad)[0])
+            raise AssertionError("step %d: %s differs at %d element(s) of a chunk; first at flat index %d: gpu=%r cpu=%r" % (
+                step, what, nbad, lo + j, float(g[j]), float(ref[j])))
+        inexact += int((g.view(torch.int32) != ref.view(torch.int32)).sum())
+        del ref, bad
+    return inexact
 
 
 def unpack_sign_bits(bits: np.ndarray, word_off: np.ndarray, block_offsets: np.ndarray) -> np.ndarray:

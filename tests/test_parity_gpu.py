@@ -230,6 +230,27 @@ def test_config5_sweep_points_oracle_sized(mode, n):
     run_workload(W.sweep_point(1 << 20, n, mode, "cuda"), steps=3)
 
 
+@pytest.mark.parametrize("mode", ["topk", "sign", "dense"])
+def test_config5_sweep_point_d_2_24_n_8_against_the_full_oracle(mode):
+    from parity import run_workload
+    run_workload(W.sweep_point(1 << 24, 8, mode, "cuda"), steps=3, check_e_every=3)
+
+
+@pytest.mark.parametrize("mode", ["topk", "sign", "dense"])
+def test_config5_largest_point_d_2_27_n_32_against_the_full_oracle(mode):
+    # the largest configuration: n d = 2^32 elements (16 GiB per [n, d] buffer), every index beyond 32 bits.
+    # Two chained steps: the first Top-k selection runs the dense passes, the second the candidate path.
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80 * (1 << 30):
+        pytest.skip("needs about 80 GiB of free device memory")
+    import psutil
+    if psutil.virtual_memory().available < 120 * (1 << 30):
+        pytest.skip("needs about 120 GiB of free host memory for the oracle")
+    from parity import run_workload
+    run_workload(W.sweep_point(1 << 27, 32, mode, "cuda"), steps=2, check_e_every=2)
+    torch.cuda.empty_cache()
+
+
 # ------------------------------------------------------------------ the candidate path and its fallbacks
 
 def _status(opt):
@@ -271,6 +292,30 @@ def test_topk_candidate_path_with_heavily_duplicated_values():
     def make(gen, t):
         return torch.randint(-20, 21, (n, d), generator=gen, device="cuda").float()
     _pair_run(n, d, [0, d], TOPK, 0.01, make, steps=6, check_e_every=2)
+
+
+def test_topk_long_list_with_thousands_of_candidates_in_the_threshold_bin():
+    # whole-vector selection over a long list whose threshold bin holds more candidates than shared
+    # memory can rank pair by pair: (a) thousands of exact duplicates of the threshold value, told apart
+    # by index only; (b) a very large k, where the bin's candidates differ in their low key bits
+    n, d = 2, 320 * 8192
+    def dup(gen, t):
+        return torch.randint(-400, 401, (n, d), generator=gen, device="cuda").float()
+    _pair_run(n, d, [0, d], TOPK, 0.01, dup, steps=5, check_e_every=2)
+    d = 48 * (1 << 20) + 13
+    p_steps = 4
+    from parity import Pair
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    p = Pair(n, d, [0, d], TOPK, 0.03)
+    try:
+        p.start(torch.zeros(d, device="cuda"))
+        for t in range(p_steps):
+            p.step(torch.randn(n, d, generator=gen, device="cuda"), check_e=(t == p_steps - 1))
+        st = _status(p.gpu)
+        assert st[0] == 0 and st[1] + st[2] == p_steps * n
+        assert st[2] >= n, "the candidate path never decided a selection: %r" % (st,)
+    finally:
+        p.close()
 
 
 def test_topk_layerwise_many_lists_single_cta_select():
