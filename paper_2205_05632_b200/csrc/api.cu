@@ -149,10 +149,14 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
         c->n_sel_small = (int)small_l.size();
         c->n_sel_big = (int)big_l.size();
         if (c->n_sel_big > 0) {
-            // enough slices for about four CTAs per SM over all long lists
+            // enough slices for about four CTAs per SM over all long lists, and short enough (about
+            // 12 K of the expected 2.5 k_b candidates each) that a slice is a few dozen loads per thread
             const int64_t lists = (int64_t)c->n * c->n_sel_big;
             int64_t parts = (4 * (int64_t)c->num_sms + lists - 1) / lists;
-            c->sel_parts = (int)(parts < 1 ? 1 : parts > 64 ? 64 : parts);
+            int64_t kb_max = 0;
+            for (int32_t sg : big_l) kb_max = std::max<int64_t>(kb_max, segs[(size_t)sg].kb);
+            parts = std::max<int64_t>(parts, (5 * kb_max / 2 + 12287) / 12288);
+            c->sel_parts = (int)(parts < 1 ? 1 : parts > 1024 ? 1024 : parts);
             RC(dev_alloc(c, &c->tk.sel_hist, (size_t)lists * kSelBins));
             RC(dev_alloc(c, &c->tk.sel_ticket, (size_t)lists * 2));
             RC(dev_alloc(c, &c->tk.sel_surv, (size_t)lists * kSurvCapBig, false));

@@ -21,6 +21,8 @@ constexpr uint32_t kNoPrediction = 0xffffffffu;  // tau_hat value that no key re
 constexpr int kTileCand = 1024;          // candidates one tile can stage in shared memory
 constexpr int kSurvCap = 1536;           // threshold-bin candidates a select can rank in shared memory
 constexpr int kSurvCapBig = 65536;       // threshold-bin candidates of a long list (kept in global memory)
+constexpr int kSurvSmem = 4096;          // ... of which this many fit the finishing CTA's shared memory
+constexpr int kRankMax = 256;            // ... and up to this many are ranked pair by pair
 constexpr int kSelBins = 4096;           // bins of the candidate select's first histogram
 constexpr int kSelectSingleMax = 24576;  // candidate capacity up to which one CTA handles a segment
 

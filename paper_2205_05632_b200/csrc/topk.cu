@@ -562,7 +562,8 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
 
 __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                 int nlist, int parts) {
-    __shared__ uint2 surv[kSurvCap];
+    __shared__ uint2 surv[kSurvSmem];
+    __shared__ uint32_t sh_hist[kThreads];
     __shared__ uint32_t scratch[kWarps];
     __shared__ uint32_t sh_base, sh_wcnt, sh_tau;
     __shared__ int is_last;
@@ -656,61 +657,61 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
     }
     const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
     uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
-    if (!take_all0 && nsurv > (uint32_t)kSurvCap) {
-        // A very long list leaves more of the threshold bin than shared memory can rank pair by pair.
-        // The survivors differ in the low S key bits and the index; the k_rem-th largest of these
-        // (low bits, lower index first) composites is found digit by digit, 8 bits at a time from
-        // the top, with a 256-bin histogram over the survivors that match the digits found so far.
-        uint32_t* hist = reinterpret_cast<uint32_t*>(surv);  // 256 words of the (here unused) ranking buffer
+    if (!take_all0 && nsurv > (uint32_t)kRankMax) {
+        // Too many candidates in the threshold bin to rank pair by pair. They differ in the low S key
+        // bits and the index; the k_rem-th largest of these (low bits, lower index first) composites
+        // is found digit by digit, 8 bits at a time from the top, with a 256-bin histogram over the
+        // candidates that match the digits found so far. The composites sit in shared memory when
+        // they fit, otherwise every pass reads the candidates again.
+        static_assert(kThreads == 256, "one histogram bin per thread");
+        unsigned long long* comp = reinterpret_cast<unsigned long long*>(surv);
+        uint32_t* hist = sh_hist;
         const uint32_t lowmask = S ? ((1u << S) - 1u) : 0u;
         auto comp_of = [&](const uint2& cv) -> unsigned long long {
             const uint32_t o = (cv.y & 0x7fffffffu) - tau_hat;
             return ((unsigned long long)(o & lowmask) << 32) | (unsigned long long)(0xffffffffu - cv.x);
         };
+        const bool in_smem = nsurv <= (uint32_t)kSurvSmem;
+        if (in_smem)
+            for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) comp[q] = comp_of(__ldcg(gsurv + q));
         unsigned long long prefix = 0ull;  // digits found so far, right-aligned
-        uint32_t need = k_rem;             // rank still to be located among the survivors matching `prefix`
+        uint32_t need = k_rem;             // rank still to be located among the candidates matching `prefix`
         const int top = ((S + 32 + 7) / 8 - 1) * 8;
         for (int shift = top; shift >= 0; shift -= 8) {
             __syncthreads();
             hist[threadIdx.x] = 0u;
             __syncthreads();
             for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
-                const unsigned long long cq = comp_of(__ldcg(gsurv + q));
+                const unsigned long long cq = in_smem ? comp[q] : comp_of(__ldcg(gsurv + q));
                 const bool match = (shift + 8 >= 64) || ((cq >> (shift + 8)) == prefix);
                 if (match) atomicAdd(&hist[(uint32_t)(cq >> shift) & 255u], 1u);
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                uint32_t above = 0;
-                int dsel = 255;
-                for (; dsel > 0; --dsel) {
-                    if (above + hist[dsel] >= need) break;
-                    above += hist[dsel];
-                }
-                sh_base = (uint32_t)dsel;
-                sh_wcnt = above;
+            // thread t looks at digit 255 - t: `incl` candidates have this digit or a larger one
+            const uint32_t hv = hist[255 - threadIdx.x];
+            uint32_t tot;
+            const uint32_t incl = block_inclusive_scan(hv, scratch, &tot);
+            if (incl - hv < need && need <= incl) {
+                sh_base = 255u - threadIdx.x;
+                sh_wcnt = incl - hv;
             }
             __syncthreads();
             prefix = (prefix << 8) | (unsigned long long)sh_base;
             need -= sh_wcnt;
         }
-        // `prefix` is now the composite of the k_rem-th largest survivor (composites are distinct)
+        // `prefix` is now the composite of the k_rem-th largest candidate (composites are distinct)
         const unsigned long long thr = prefix;
         tau = tau_hat + (uint32_t)(((unsigned long long)b0 << S) | (thr >> 32));
-        for (uint32_t q0 = 0; q0 < nsurv; q0 += kThreads) {  // uniform trip count: the loop holds barriers
-            const uint32_t q = q0 + threadIdx.x;
-            uint2 cv = make_uint2(0u, 0u);
-            bool kept = false;
-            if (q < nsurv) {
-                cv = __ldcg(gsurv + q);
-                kept = comp_of(cv) >= thr;
-            }
-            uint32_t tot3;
-            const uint32_t incl = block_inclusive_scan(kept ? 1u : 0u, scratch, &tot3);
-            if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
-            __syncthreads();
-            if (kept) {
-                const uint32_t pos = sh_base + incl - 1u;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            sh_base = atomicAdd(&st->emit_count, k_rem);
+            sh_wcnt = 0u;
+        }
+        __syncthreads();
+        for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) {
+            const uint2 cv = __ldcg(gsurv + q);
+            if (comp_of(cv) >= thr) {
+                const uint32_t pos = sh_base + atomicAdd(&sh_wcnt, 1u);
                 if (pos < kb) {
                     b.idx[slot0 + pos] = (int32_t)cv.x;
                     b.val[slot0 + pos] = __uint_as_float(cv.y);
@@ -718,8 +719,9 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
                     atomicOr(b.status, 1u);
                 }
             }
-            __syncthreads();
         }
+        __syncthreads();
+        if (threadIdx.x == 0 && sh_wcnt != k_rem) atomicOr(b.status, 1u);
     } else if (!take_all0) {
         for (uint32_t q = threadIdx.x; q < nsurv; q += kThreads) surv[q] = __ldcg(gsurv + q);
         __syncthreads();
