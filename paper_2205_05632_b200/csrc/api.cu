@@ -380,6 +380,7 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
     c->hp.omb2 = 1.0f - beta2;
     c->hp.eps = eps;
     c->hp.nf = (float)n;
+    c->hp.inv_nf = ((n & (n - 1)) == 0) ? 1.0f / (float)n : 0.0f;
     int rc;
     try {
         rc = init_context(c, block_offsets);

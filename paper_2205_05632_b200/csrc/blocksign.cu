@@ -252,8 +252,8 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
     a2 = all - (a2 + a2);
     a3 = all - (a3 + a3);
     if (r >= len) return;
-    const float gb[4] = {mean_from_acc(a0, hp.nf), mean_from_acc(a1, hp.nf), mean_from_acc(a2, hp.nf),
-                         mean_from_acc(a3, hp.nf)};
+    const float gb[4] = {mean_from_acc(a0, hp), mean_from_acc(a1, hp), mean_from_acc(a2, hp),
+                         mean_from_acc(a3, hp)};
     if (full) {
         amsgrad_update(gb[0], mm.x, vv.x, hh.x, tt.x, hp);
         amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);

@@ -52,6 +52,7 @@ struct SegParams {
 // AMSGrad hyper-parameters as the fp32 numbers every kernel uses (Algorithm 1).
 struct HyperParams {
     float lr, beta1, beta2, omb1, omb2, eps, nf;  // omb = 1 - beta (fp32), nf = (float)n
+    float inv_nf;  // 1 / n when n is a power of two (then x * inv_nf == x / n bit for bit), else 0
 };
 
 // One AMSGrad coordinate update (Algorithm 2, lines 13-16). Every operation is a separately
@@ -65,8 +66,12 @@ __device__ __forceinline__ void amsgrad_update(float g, float& m, float& v, floa
 }
 
 // gbar = (float)(sum over workers, accumulated in binary64) / (float)n  (Algorithm 2, line 12).
-__device__ __forceinline__ float mean_from_acc(double acc, float nf) {
-    return __fdiv_rn(__double2float_rn(acc), nf);
+// For n a power of two the division is a multiplication by the exactly representable 1 / n: both
+// round the same real number once, so the bits agree (subnormal results included) and the
+// multi-instruction IEEE division is saved.
+__device__ __forceinline__ float mean_from_acc(double acc, const HyperParams& hp) {
+    const float s = __double2float_rn(acc);
+    return hp.inv_nf != 0.0f ? __fmul_rn(s, hp.inv_nf) : __fdiv_rn(s, hp.nf);
 }
 
 // Magnitude key: fp32 bits with the sign cleared; unsigned order == order of |x| for finite x.

@@ -31,8 +31,8 @@ __global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t
             a2 += (double)g.z;
             a3 += (double)g.w;
         }
-        float4 gb = make_float4(mean_from_acc(a0, hp.nf), mean_from_acc(a1, hp.nf), mean_from_acc(a2, hp.nf),
-                                mean_from_acc(a3, hp.nf));
+        float4 gb = make_float4(mean_from_acc(a0, hp), mean_from_acc(a1, hp), mean_from_acc(a2, hp),
+                                mean_from_acc(a3, hp));
         float4 mm = *reinterpret_cast<const float4*>(m + j);
         float4 vv = *reinterpret_cast<const float4*>(v + j);
         float4 vh = *reinterpret_cast<const float4*>(vhat + j);
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t
         const int64_t j = (groups << 2) + threadIdx.x;
         double a = 0.0;
         for (int32_t i = 0; i < n; ++i) a += (double)G[(size_t)i * (size_t)d + (size_t)j];
-        float gb = mean_from_acc(a, hp.nf);
+        float gb = mean_from_acc(a, hp);
         float mm = m[j], vv = v[j], vh = vhat[j], th = theta[j];
         amsgrad_update(gb, mm, vv, vh, th, hp);
         gbar[j] = gb;
@@ -118,8 +118,8 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
             *reinterpret_cast<double2*>(b.acc + j) = make_double2(0.0, 0.0);
             *reinterpret_cast<double2*>(b.acc + j + 2) = make_double2(0.0, 0.0);
         }
-        float4 gb = make_float4(mean_from_acc(a[0], hp.nf), mean_from_acc(a[1], hp.nf), mean_from_acc(a[2], hp.nf),
-                                mean_from_acc(a[3], hp.nf));
+        float4 gb = make_float4(mean_from_acc(a[0], hp), mean_from_acc(a[1], hp), mean_from_acc(a[2], hp),
+                                mean_from_acc(a[3], hp));
         amsgrad_update(gb.x, mm.x, vv.x, vh.x, th.x, hp);
         amsgrad_update(gb.y, mm.y, vv.y, vh.y, th.y, hp);
         amsgrad_update(gb.z, mm.z, vv.z, vh.z, th.z, hp);
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
                 ak += b.acc[j + k];
                 b.acc[j + k] = 0.0;
             }
-            const float gb = mean_from_acc(ak, hp.nf);
+            const float gb = mean_from_acc(ak, hp);
             float m1 = b.m[j + k], v1 = b.v[j + k], h1 = b.vhat[j + k], t1 = theta[j + k];
             amsgrad_update(gb, m1, v1, h1, t1, hp);
             b.gbar[j + k] = gb;
