@@ -149,6 +149,42 @@ int compams_step(compams_handle h, const float* grads, float* theta);
  */
 int compams_step_host(compams_handle h, const float* grads_host, float* theta_host);
 
+/*
+ * Workers sharded over several handles (several GPUs or processes), as in Algorithm 2 proper: every
+ * worker compresses locally and "sends g~_{t,i} to the central server" (line 9); the server averages
+ * the n compressed gradients and updates theta (lines 11-16). Here every shard also plays the server
+ * on its own replica of theta, m, v, vhat: after the shards have exchanged their compressed gradients
+ * (an all-gather of the message buffers - the only communication, and it is the caller's: this library
+ * starts no collective), each applies the identical update, so the replicas stay bit-identical and
+ * theta needs no broadcast.
+ *
+ * compams_create_sharded - like compams_create, for a handle that holds workers first_worker ...
+ *   first_worker + n_local - 1 of n_total (1 <= n_local, first_worker >= 0,
+ *   first_worker + n_local <= n_total <= 65535). E is [n_local, d]; the message buffers
+ *   (BUF_TOPK_IDX / BUF_TOPK_VAL [n_total, K], or BUF_SIGN_BITS [n_total, W] and BUF_SCALES
+ *   [n_total, M]) have one row per worker of the whole job. The uncompressed mode (every k_b = d_b)
+ *   has no message to exchange and is refused (INVALID_ARG). compams_create(n, ...) is
+ *   compams_create_sharded(n, n, 0, ...).
+ *
+ * compams_compress - lines 5-9 for this handle's workers: x = g + e, the compression, the residual.
+ *   grads   device; [n_local, d] fp32 packed, 4-byte aligned; read only.
+ *   Fills rows first_worker ... first_worker + n_local - 1 of the message buffers. The caller then
+ *   makes the other rows hold the other shards' messages (for Block-Sign BUF_SCALES must be asked for
+ *   AFTER this call: two scale buffers alternate), ordered on the handle's stream before compams_apply.
+ *
+ * compams_apply - lines 11-16: gbar_t = (1/n_total) sum of the n_total messages, then the AMSGrad update.
+ *   theta   device; [d] fp32, 16-byte aligned; updated in place.
+ *
+ * compams_step on a handle with n_local == n_total is compams_compress followed by compams_apply;
+ * on a sharded handle it returns INVALID_ARG (the exchange is missing). Both calls enqueue on the
+ * handle's stream and return without synchronising.
+ */
+int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total, int32_t first_worker, int64_t d,
+                           const int64_t* block_offsets, int32_t num_blocks, int32_t compressor, double k_ratio, float lr,
+                           float beta1, float beta2, float eps);
+int compams_compress(compams_handle h, const float* grads);
+int compams_apply(compams_handle h, float* theta);
+
 /* compams_destroy - free everything the handle owns (synchronises its stream first).
  * A null handle is a no-op. */
 int compams_destroy(compams_handle h);

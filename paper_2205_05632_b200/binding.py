@@ -68,6 +68,13 @@ def load_library() -> ctypes.CDLL:
     L.compams_step.argtypes = [H, c.c_void_p, c.c_void_p]
     L.compams_step_host.restype = c.c_int
     L.compams_step_host.argtypes = [H, c.c_void_p, c.c_void_p]
+    L.compams_create_sharded.restype = c.c_int
+    L.compams_create_sharded.argtypes = [c.POINTER(H), c.c_int32, c.c_int32, c.c_int32, c.c_int64, c.POINTER(c.c_int64),
+                                         c.c_int32, c.c_int32, c.c_double, c.c_float, c.c_float, c.c_float, c.c_float]
+    L.compams_compress.restype = c.c_int
+    L.compams_compress.argtypes = [H, c.c_void_p]
+    L.compams_apply.restype = c.c_int
+    L.compams_apply.argtypes = [H, c.c_void_p]
     L.compams_destroy.restype = c.c_int
     L.compams_destroy.argtypes = [H]
     L.compams_set_stream.restype = c.c_int
@@ -161,19 +168,25 @@ class CompAMS:
 
     def __init__(self, n: int, d: int, block_offsets: Sequence[int], compressor: int, k_ratio: float = 1.0,
                  lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, n_total: Optional[int] = None, first_worker: int = 0):
+        """`n` workers live in this optimizer. With `n_total` > n they are workers `first_worker` ...
+        `first_worker + n - 1` of a job whose other workers live in other optimizers (other GPUs): use
+        compress() / apply() with an exchange of the message buffers in between instead of step()."""
         self._L = load_library()
         self.n, self.d = int(n), int(d)
+        self.n_total = self.n if n_total is None else int(n_total)
+        self.first_worker = int(first_worker)
         offs = np.ascontiguousarray(block_offsets, dtype=np.int64)
         self.M = int(offs.size - 1)
         self.compressor = int(compressor)
         self._h = ctypes.c_void_p()
-        rc = self._L.compams_create(ctypes.byref(self._h), self.n, self.d,
-                                    offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), self.M, self.compressor,
-                                    float(k_ratio), float(lr), float(beta1), float(beta2), float(eps))
+        rc = self._L.compams_create_sharded(ctypes.byref(self._h), self.n, self.n_total, self.first_worker, self.d,
+                                            offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), self.M,
+                                            self.compressor, float(k_ratio), float(lr), float(beta1), float(beta2),
+                                            float(eps))
         if rc != 0:
             self._h = ctypes.c_void_p()
-        _check(rc, "compams_create")
+        _check(rc, "compams_create_sharded")
         self.set_stream(stream if stream is not None else torch.cuda.current_stream())
 
     # -- calls ---------------------------------------------------------------------------------
@@ -224,6 +237,26 @@ class CompAMS:
         _check(self._L.compams_step(self._h, ctypes.c_void_p(grads.data_ptr()), ctypes.c_void_p(theta.data_ptr())),
                "compams_step")
 
+    def compress(self, grads: torch.Tensor) -> None:
+        """Worker side of one iteration (Algorithm 2, lines 5-9) for this optimizer's workers."""
+        if not (grads.is_cuda and grads.dtype == torch.float32 and grads.is_contiguous()
+                and tuple(grads.shape) == (self.n, self.d)):
+            raise CompAMSError("grads must be a contiguous float32 CUDA tensor of shape [n, d]")
+        _check(self._L.compams_compress(self._h, ctypes.c_void_p(grads.data_ptr())), "compams_compress")
+
+    def apply(self, theta: torch.Tensor) -> None:
+        """Server side (lines 11-16) over the messages of all n_total workers."""
+        if not (theta.is_cuda and theta.dtype == torch.float32 and theta.is_contiguous()
+                and tuple(theta.shape) == (self.d,)):
+            raise CompAMSError("theta must be a contiguous float32 CUDA tensor of shape [d]")
+        _check(self._L.compams_apply(self._h, ctypes.c_void_p(theta.data_ptr())), "compams_apply")
+
+    def message_buffers(self):
+        """The buffers an exchange between shards has to complete, as [n_total, width] views: every
+        shard has filled rows first_worker ... first_worker + n - 1. Ask after compress()."""
+        names = ("topk_idx", "topk_val") if self.compressor == TOPK else ("sign_bits", "scales")
+        return [self.buffer(name) for name in names]
+
     def step_host(self, grads: torch.Tensor, theta: torch.Tensor) -> None:
         if grads.is_cuda or theta.is_cuda:
             raise CompAMSError("step_host() takes host tensors")
@@ -250,9 +283,9 @@ class CompAMS:
         if name == "E":
             return t.view(self.n, self.d)
         if name in ("topk_idx", "topk_val", "sign_bits"):
-            return t.view(self.n, -1)
+            return t.view(self.n_total, -1)
         if name == "scales":
-            return t.view(self.n, self.M)
+            return t.view(self.n_total, self.M)
         return t
 
     def check_status(self) -> int:

@@ -213,8 +213,10 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_upload(c, &d_small, small));
         t.small_blk = d_small;
         t.nsmall = (int32_t)small.size();
-        RC(dev_alloc(c, &t.idx, (size_t)n * (size_t)c->K));
-        RC(dev_alloc(c, &t.val, (size_t)n * (size_t)c->K));
+        // the messages of all n_total workers: this handle's selection fills its own rows, the other
+        // rows are filled by the caller's exchange before compams_apply
+        RC(dev_alloc(c, &t.idx, (size_t)c->n_total * (size_t)c->K));
+        RC(dev_alloc(c, &t.val, (size_t)c->n_total * (size_t)c->K));
         RC(dev_alloc(c, &t.hist, (size_t)n * (size_t)c->tab.nseg * kBins1));
         {
             SegState init{};
@@ -241,9 +243,9 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
             // kept entries are handed to the server grouped by coordinate range: room for four times the
             // average load of a bucket, the rare excess goes through the binary64 accumulator
             t.nbucket = (int32_t)((d + kBucketSpan - 1) / kBucketSpan);
-            const int64_t avg = ((int64_t)n * c->K + t.nbucket - 1) / t.nbucket;
+            const int64_t avg = ((int64_t)c->n_total * c->K + t.nbucket - 1) / t.nbucket;
             int64_t cap = 4 * avg + 64;
-            if (cap > (int64_t)n * kBucketSpan) cap = (int64_t)n * kBucketSpan;
+            if (cap > (int64_t)c->n_total * kBucketSpan) cap = (int64_t)c->n_total * kBucketSpan;
             t.bucket_cap = (int32_t)((cap + 31) / 32 * 32);
             RC(dev_alloc(c, &t.bucket, (size_t)t.nbucket * (size_t)t.bucket_cap, false));
             RC(dev_alloc(c, &t.bcount, (size_t)t.nbucket));
@@ -270,9 +272,10 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         s.E = c->E;
         s.word_off = c->d_word_off;
         s.W = c->W;
-        RC(dev_alloc(c, &s.bits, (size_t)n * (size_t)c->W));
-        RC(dev_alloc(c, &c->scales[0], (size_t)n * (size_t)M));
-        RC(dev_alloc(c, &c->scales[1], (size_t)n * (size_t)M));
+        // sign words and scales of all n_total workers (see the Top-k messages above)
+        RC(dev_alloc(c, &s.bits, (size_t)c->n_total * (size_t)c->W));
+        RC(dev_alloc(c, &c->scales[0], (size_t)c->n_total * (size_t)M));
+        RC(dev_alloc(c, &c->scales[1], (size_t)c->n_total * (size_t)M));
         RC(dev_alloc(c, &s.tile_sum, (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &s.edge, (size_t)n * (size_t)c->tab.ntiles));
         s.gbar = c->gbar;
@@ -319,17 +322,15 @@ int run_kernel(compams_context* c, int kernel, F&& launch) {
     return COMPAMS_OK;
 }
 
-int step_device(compams_context* c, const float* grads, float* theta) {
+// Worker side of one iteration (Algorithm 2, lines 5-9) for this handle's workers: x = g + e, the
+// compression, the residual; the compressed gradients land in this handle's rows of the message buffers.
+int compress_device(compams_context* c, const float* grads) {
     ++c->steps_done;
-    if (c->compressor == COMPAMS_TOPK && c->identity) {
-        return run_kernel(c, COMPAMS_K_DENSE_MEAN_AMSGRAD, [&] { return launch_dense_mean_amsgrad(c, grads, theta); });
-    }
     if (c->compressor == COMPAMS_BLOCKSIGN) {
         c->scales_cur ^= 1;
         RC(run_kernel(c, COMPAMS_K_BS_SWEEP, [&] { return launch_bs_sweep(c, grads); }));
         c->e_is_x = true;
         RC(run_kernel(c, COMPAMS_K_BS_SCALES, [&] { return launch_bs_scales(c); }));
-        RC(run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); }));
         return COMPAMS_OK;
     }
     // kept coordinates are recorded in a bit map; their e is zeroed when E is next read (by the next
@@ -344,20 +345,34 @@ int step_device(compams_context* c, const float* grads, float* theta) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SELECT, [&] { return launch_topk_select(c); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_DENSE, [&] { return launch_topk_dense(c); }));
     }
+    return COMPAMS_OK;
+}
+
+// Server side (Algorithm 2, lines 11-16): average of the n_total compressed gradients and AMSGrad.
+int apply_device(compams_context* c, float* theta) {
+    if (c->compressor == COMPAMS_BLOCKSIGN) {
+        return run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); });
+    }
     RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c); }));
     c->e_mask_pending = true;
     RC(run_kernel(c, COMPAMS_K_AMSGRAD, [&] { return launch_amsgrad(c, theta); }));
     return COMPAMS_OK;
 }
 
-}  // namespace
+int step_device(compams_context* c, const float* grads, float* theta) {
+    if (c->compressor == COMPAMS_TOPK && c->identity) {
+        ++c->steps_done;
+        return run_kernel(c, COMPAMS_K_DENSE_MEAN_AMSGRAD, [&] { return launch_dense_mean_amsgrad(c, grads, theta); });
+    }
+    RC(compress_device(c, grads));
+    return apply_device(c, theta);
+}
 
-extern "C" {
-
-int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* block_offsets, int32_t num_blocks,
-                   int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps) {
+int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0, int64_t d, const int64_t* block_offsets,
+                  int32_t num_blocks, int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps) {
     if (!out || !block_offsets) return COMPAMS_ERR_INVALID_ARG;
-    if (n < 1 || n > 65535 || d < 1 || d >= ((int64_t)1 << 31) || num_blocks < 1 || (int64_t)num_blocks > d)
+    if (n < 1 || n_total > 65535 || row0 < 0 || (int64_t)row0 + n > n_total || d < 1 || d >= ((int64_t)1 << 31) ||
+        num_blocks < 1 || (int64_t)num_blocks > d)
         return COMPAMS_ERR_INVALID_ARG;
     if (compressor != COMPAMS_TOPK && compressor != COMPAMS_BLOCKSIGN) return COMPAMS_ERR_INVALID_ARG;
     if (compressor == COMPAMS_TOPK && !(k_ratio > 0.0 && k_ratio <= 1.0)) return COMPAMS_ERR_INVALID_ARG;
@@ -369,6 +384,8 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
     compams_context* c = new (std::nothrow) compams_context();
     if (!c) return COMPAMS_ERR_ALLOC;
     c->n = n;
+    c->n_total = n_total;
+    c->row0 = row0;
     c->d = d;
     c->M = num_blocks;
     c->compressor = compressor;
@@ -379,14 +396,16 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
     c->hp.omb1 = 1.0f - beta1;
     c->hp.omb2 = 1.0f - beta2;
     c->hp.eps = eps;
-    c->hp.nf = (float)n;
-    c->hp.inv_nf = ((n & (n - 1)) == 0) ? 1.0f / (float)n : 0.0f;
+    c->hp.nf = (float)n_total;
+    c->hp.inv_nf = ((n_total & (n_total - 1)) == 0) ? 1.0f / (float)n_total : 0.0f;
     int rc;
     try {
         rc = init_context(c, block_offsets);
     } catch (const std::bad_alloc&) {
         rc = COMPAMS_ERR_ALLOC;
     }
+    // sharded workers exchange compressed gradients; the uncompressed mode (k = d) has none to exchange
+    if (!rc && n != n_total && c->identity) rc = COMPAMS_ERR_INVALID_ARG;
     if (rc) {
         free_context(c);
         return rc;
@@ -395,10 +414,47 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
     return COMPAMS_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* block_offsets, int32_t num_blocks,
+                   int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps) {
+    return create_handle(out, n, n, 0, d, block_offsets, num_blocks, compressor, k_ratio, lr, beta1, beta2, eps);
+}
+
+int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total, int32_t first_worker, int64_t d,
+                           const int64_t* block_offsets, int32_t num_blocks, int32_t compressor, double k_ratio, float lr,
+                           float beta1, float beta2, float eps) {
+    return create_handle(out, n_local, n_total, first_worker, d, block_offsets, num_blocks, compressor, k_ratio, lr, beta1,
+                         beta2, eps);
+}
+
+int compams_compress(compams_handle c, const float* grads) {
+    if (!c || !grads || (reinterpret_cast<uintptr_t>(grads) & 3u)) return COMPAMS_ERR_INVALID_ARG;
+    if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;  // k = d: nothing is compressed
+    try {
+        return compress_device(c, grads);
+    } catch (const std::bad_alloc&) {
+        return COMPAMS_ERR_ALLOC;
+    }
+}
+
+int compams_apply(compams_handle c, float* theta) {
+    if (!c || !theta || (reinterpret_cast<uintptr_t>(theta) & 15u)) return COMPAMS_ERR_INVALID_ARG;
+    if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;
+    try {
+        return apply_device(c, theta);
+    } catch (const std::bad_alloc&) {
+        return COMPAMS_ERR_ALLOC;
+    }
+}
+
 int compams_step(compams_handle c, const float* grads, float* theta) {
     if (!c || !grads || !theta) return COMPAMS_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(grads) & 3u) || (reinterpret_cast<uintptr_t>(theta) & 15u))
         return COMPAMS_ERR_INVALID_ARG;
+    if (c->n != c->n_total) return COMPAMS_ERR_INVALID_ARG;  // the other workers' messages have to be exchanged first
     try {
         return step_device(c, grads, theta);
     } catch (const std::bad_alloc&) {
@@ -407,7 +463,7 @@ int compams_step(compams_handle c, const float* grads, float* theta) {
 }
 
 int compams_step_host(compams_handle c, const float* grads_host, float* theta_host) {
-    if (!c || !grads_host || !theta_host) return COMPAMS_ERR_INVALID_ARG;
+    if (!c || !grads_host || !theta_host || c->n != c->n_total) return COMPAMS_ERR_INVALID_ARG;
     const size_t gbytes = (size_t)c->n * (size_t)c->d * sizeof(float);
     const size_t tbytes = (size_t)c->d * sizeof(float);
     if (!c->stage_grads) {
@@ -542,12 +598,12 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
         case COMPAMS_BUF_V: p = c->v; cnt = c->d; break;
         case COMPAMS_BUF_VHAT: p = c->vhat; cnt = c->d; break;
         case COMPAMS_BUF_GBAR: p = c->gbar; cnt = c->d; break;
-        case COMPAMS_BUF_TOPK_IDX: if (topk) { p = c->tk.idx; cnt = (int64_t)c->n * c->K; } break;
-        case COMPAMS_BUF_TOPK_VAL: if (topk) { p = c->tk.val; cnt = (int64_t)c->n * c->K; } break;
+        case COMPAMS_BUF_TOPK_IDX: if (topk) { p = c->tk.idx; cnt = (int64_t)c->n_total * c->K; } break;
+        case COMPAMS_BUF_TOPK_VAL: if (topk) { p = c->tk.val; cnt = (int64_t)c->n_total * c->K; } break;
         case COMPAMS_BUF_TOPK_SEG_OFFSETS: if (topk) { p = c->d_seg_off; cnt = c->M + 1; } break;
-        case COMPAMS_BUF_SIGN_BITS: if (sign) { p = c->bs.bits; cnt = (int64_t)c->n * c->W; } break;
+        case COMPAMS_BUF_SIGN_BITS: if (sign) { p = c->bs.bits; cnt = (int64_t)c->n_total * c->W; } break;
         case COMPAMS_BUF_SIGN_WORD_OFFSETS: if (sign) { p = c->d_word_off; cnt = c->M + 1; } break;
-        case COMPAMS_BUF_SCALES: if (sign) { p = c->scales[c->scales_cur]; cnt = (int64_t)c->n * c->M; } break;
+        case COMPAMS_BUF_SCALES: if (sign) { p = c->scales[c->scales_cur]; cnt = (int64_t)c->n_total * c->M; } break;
         case COMPAMS_BUF_STATUS: p = c->status; cnt = 8; break;
         default: return COMPAMS_ERR_INVALID_ARG;
     }

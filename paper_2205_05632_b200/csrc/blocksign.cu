@@ -280,32 +280,45 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
     }
 }
 
+// The worker-side kernels see this handle's own rows of the message buffers (sign words, scales);
+// the server kernel sees the rows of all n_total workers.
+static BsBuffers own_rows(const compams_context* c) {
+    BsBuffers b = c->bs;
+    const size_t r0 = (size_t)c->row0;
+    b.bits = c->bs.bits + r0 * (size_t)c->W;
+    b.scales_prev = c->scales[c->scales_cur ^ 1] + r0 * (size_t)c->M;
+    b.scales_cur = c->scales[c->scales_cur] + r0 * (size_t)c->M;
+    return b;
+}
+
 cudaError_t launch_bs_sweep(compams_context* c, const float* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    BsBuffers b = c->bs;
-    b.scales_prev = c->scales[c->scales_cur ^ 1];
-    b.scales_cur = c->scales[c->scales_cur];
-    bs_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, grads, c->e_is_x ? 1 : 0, c->segp);
+    bs_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), grads, c->e_is_x ? 1 : 0, c->segp);
     return cudaGetLastError();
 }
 
 cudaError_t launch_bs_scales(compams_context* c) {
     dim3 grid((unsigned)c->M, (unsigned)c->n);
-    BsBuffers b = c->bs;
-    b.scales_cur = c->scales[c->scales_cur];
-    return launch_after(bs_scales_kernel, grid, dim3(kThreads), c->stream, c->tab, b);
+    return launch_after(bs_scales_kernel, grid, dim3(kThreads), c->stream, c->tab, own_rows(c));
 }
 
 cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     BsBuffers b = c->bs;
     b.scales_cur = c->scales[c->scales_cur];
-    return launch_after(bs_apply_kernel, dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), c->stream, c->tab, b,
-                        theta, c->hp, c->segp);
+    Tables t = c->tab;
+    t.n = c->n_total;  // the average runs over every worker's message
+    if (c->n == c->n_total)
+        return launch_after(bs_apply_kernel, dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), c->stream, t, b, theta,
+                            c->hp, c->segp);
+    // sharded workers: the other workers' messages were written by the caller's exchange, which is
+    // ordered on the stream like any kernel; a plain launch waits for it
+    bs_apply_kernel<<<dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_bs_materialize(compams_context* c) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    bs_materialize_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->E, c->scales[c->scales_cur]);
+    bs_materialize_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->E, c->scales[c->scales_cur] + (size_t)c->row0 * (size_t)c->M);
     return cudaGetLastError();
 }
 

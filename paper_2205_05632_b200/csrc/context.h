@@ -106,7 +106,9 @@ struct TopkBuffers {
 
 struct compams_context {
     int device = 0;
-    int32_t n = 0;
+    int32_t n = 0;        // workers whose gradients and error accumulators this handle holds
+    int32_t n_total = 0;  // workers the server averages over (> n when the workers are sharded over several handles)
+    int32_t row0 = 0;     // index of this handle's first worker among the n_total
     int64_t d = 0;
     int32_t M = 0;
     int32_t compressor = 0;

@@ -1152,7 +1152,7 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 // scatter: acc[j] += x_ij over all kept (i, j); binary64 atomics, exact hence order-independent.
 // The same walk zeroes e at the kept coordinates (they were left holding x by the sweep).
 
-__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count) {
+__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count, int32_t row0) {
     allow_dependents();
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     // the first n * nseg threads also close the step for one large-block segment each: exactly k_b
@@ -1195,7 +1195,11 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
         b.bdirty[T] = 1u;
     }
     // the coordinate's e becomes 0 (line 8: e = x - x): recorded in the kept map, applied when E is next read
-    const int64_t f = (p / b.K) * t.d + j;  // the element's index in E, [n, d] flattened
+    // (`count` covers the messages of every worker the server averages over; E and the kept map hold
+    // the t.n workers of this handle, whose first is worker row0)
+    const int64_t il = p / b.K - row0;
+    if (il < 0 || il >= t.n) return;
+    const int64_t f = il * t.d + j;  // the element's index in E, [n, d] flattened
     atomicOr(b.kept_cur + (size_t)(f >> 5), 1u << (uint32_t)(f & 31));
 }
 
@@ -1216,31 +1220,41 @@ __global__ void __launch_bounds__(kThreads) topk_materialize_kernel(int64_t nd, 
 
 // ------------------------------------------------------------------------------------------
 
+// The selection kernels see this handle's own rows of the message buffers; the server-side
+// kernels see the rows of all n_total workers.
+static TopkBuffers own_rows(const compams_context* c) {
+    TopkBuffers b = c->tk;
+    b.idx = c->tk.idx + (size_t)c->row0 * (size_t)c->K;
+    b.val = c->tk.val + (size_t)c->row0 * (size_t)c->K;
+    return b;
+}
+
 cudaError_t launch_topk_small(compams_context* c, const float* grads) {
     dim3 grid((unsigned)c->tk.nsmall, (unsigned)c->n);
-    topk_small_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, grads);
+    topk_small_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), grads);
     return cudaGetLastError();
 }
 
 cudaError_t launch_topk_sweep(compams_context* c, const float* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    topk_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, grads, c->segp);
+    topk_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), grads, c->segp);
     return cudaGetLastError();
 }
 
 cudaError_t launch_topk_select(compams_context* c) {
     cudaError_t e = cudaSuccess;
+    const TopkBuffers b = own_rows(c);
     if (c->n_sel_small > 0) {
         topk_select_kernel<<<(unsigned)((int64_t)c->n * c->n_sel_small), kSelThreads, 0, c->stream>>>(
-            c->tab, c->tk, c->sel_small, c->n_sel_small);
+            c->tab, b, c->sel_small, c->n_sel_small);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess || c->n_sel_big == 0) return e;
     const unsigned grid = (unsigned)((int64_t)c->n * c->n_sel_big * c->sel_parts);
-    topk_selhist_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, c->sel_big, c->n_sel_big, c->sel_parts);
+    topk_selhist_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, c->sel_big, c->n_sel_big, c->sel_parts);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    topk_selemit_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, c->sel_big, c->n_sel_big, c->sel_parts);
+    topk_selemit_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, c->sel_big, c->n_sel_big, c->sel_parts);
     return cudaGetLastError();
 }
 
@@ -1252,7 +1266,8 @@ cudaError_t launch_topk_dense(compams_context* c) {
         if (per_sm < 1) return cudaErrorLaunchOutOfResources;
         c->dense_grid = per_sm * c->num_sms;  // every CTA resident at once, as a cooperative launch requires
     }
-    void* args[] = {(void*)&c->tab, (void*)&c->tk};
+    TopkBuffers b = own_rows(c);
+    void* args[] = {(void*)&c->tab, (void*)&b};
     return cudaLaunchCooperativeKernel((const void*)topk_dense_kernel, dim3((unsigned)c->dense_grid), dim3(kThreads), args,
                                        0, c->stream);
 }
@@ -1265,9 +1280,10 @@ cudaError_t launch_topk_materialize(compams_context* c) {
 }
 
 cudaError_t launch_topk_scatter(compams_context* c) {
-    const int64_t count = (int64_t)c->n * c->K;  // >= n * nseg: every block keeps at least one entry
+    // one thread per message entry of every worker (>= n * nseg: every block keeps at least one entry)
+    const int64_t count = (int64_t)c->n_total * c->K;
     const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
-    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count);
+    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, c->row0);
     return cudaGetLastError();
 }
 
