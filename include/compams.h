@@ -136,6 +136,20 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
 int compams_step(compams_handle h, const float* grads, float* theta);
 
 /*
+ * compams_step_bf16 / compams_compress_bf16 - compams_step / compams_compress for gradients stored as
+ * bfloat16 (what a mixed-precision backward pass produces): the worker-side read of g shrinks from 4 to
+ * 2 bytes per element, everything else is unchanged. Line 7 of Algorithm 2 becomes x = widen(g) + e with
+ * widen exact, so the step equals compams_step on the fp32 tensor that holds the same values, bit for bit;
+ * e, the messages and the server state stay fp32. A handle may be fed fp32 in one step and bfloat16 in
+ * the next.
+ *
+ *   grads_bf16   device; [n, d] bfloat16 (16-bit patterns: sign, 8 exponent bits, 7 fraction bits), packed
+ *                row-major, 2-byte aligned; read only.
+ */
+int compams_step_bf16(compams_handle h, const void* grads_bf16, float* theta);
+int compams_compress_bf16(compams_handle h, const void* grads_bf16);
+
+/*
  * compams_step_host - the same iteration for callers whose tensors live in HOST memory
  * (Algorithm 2's "send g~ to the server / receive theta" endpoints on a machine where the
  * gradients are produced off-GPU).

@@ -66,6 +66,10 @@ def load_library() -> ctypes.CDLL:
                                  c.c_double, c.c_float, c.c_float, c.c_float, c.c_float]
     L.compams_step.restype = c.c_int
     L.compams_step.argtypes = [H, c.c_void_p, c.c_void_p]
+    L.compams_step_bf16.restype = c.c_int
+    L.compams_step_bf16.argtypes = [H, c.c_void_p, c.c_void_p]
+    L.compams_compress_bf16.restype = c.c_int
+    L.compams_compress_bf16.argtypes = [H, c.c_void_p]
     L.compams_step_host.restype = c.c_int
     L.compams_step_host.argtypes = [H, c.c_void_p, c.c_void_p]
     L.compams_create_sharded.restype = c.c_int
@@ -228,21 +232,26 @@ class CompAMS:
     def step(self, grads: torch.Tensor, theta: torch.Tensor) -> None:
         if not (grads.is_cuda and theta.is_cuda):
             raise CompAMSError("step() takes CUDA tensors; use step_host() for host tensors")
-        if grads.dtype != torch.float32 or theta.dtype != torch.float32:
-            raise CompAMSError("grads and theta must be float32")
+        if grads.dtype not in (torch.float32, torch.bfloat16) or theta.dtype != torch.float32:
+            raise CompAMSError("grads must be float32 or bfloat16, theta float32")
         if tuple(grads.shape) != (self.n, self.d) or not grads.is_contiguous():
             raise CompAMSError("grads must be a contiguous [n, d] tensor")
         if tuple(theta.shape) != (self.d,) or not theta.is_contiguous():
             raise CompAMSError("theta must be a contiguous [d] tensor")
+        if grads.dtype == torch.bfloat16:
+            _check(self._L.compams_step_bf16(self._h, ctypes.c_void_p(grads.data_ptr()),
+                                             ctypes.c_void_p(theta.data_ptr())), "compams_step_bf16")
+            return
         _check(self._L.compams_step(self._h, ctypes.c_void_p(grads.data_ptr()), ctypes.c_void_p(theta.data_ptr())),
                "compams_step")
 
     def compress(self, grads: torch.Tensor) -> None:
         """Worker side of one iteration (Algorithm 2, lines 5-9) for this optimizer's workers."""
-        if not (grads.is_cuda and grads.dtype == torch.float32 and grads.is_contiguous()
+        if not (grads.is_cuda and grads.dtype in (torch.float32, torch.bfloat16) and grads.is_contiguous()
                 and tuple(grads.shape) == (self.n, self.d)):
-            raise CompAMSError("grads must be a contiguous float32 CUDA tensor of shape [n, d]")
-        _check(self._L.compams_compress(self._h, ctypes.c_void_p(grads.data_ptr())), "compams_compress")
+            raise CompAMSError("grads must be a contiguous float32 or bfloat16 CUDA tensor of shape [n, d]")
+        fn = self._L.compams_compress_bf16 if grads.dtype == torch.bfloat16 else self._L.compams_compress
+        _check(fn(self._h, ctypes.c_void_p(grads.data_ptr())), "compams_compress")
 
     def apply(self, theta: torch.Tensor) -> None:
         """Server side (lines 11-16) over the messages of all n_total workers."""

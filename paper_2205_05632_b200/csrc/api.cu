@@ -324,7 +324,7 @@ int run_kernel(compams_context* c, int kernel, F&& launch) {
 
 // Worker side of one iteration (Algorithm 2, lines 5-9) for this handle's workers: x = g + e, the
 // compression, the residual; the compressed gradients land in this handle's rows of the message buffers.
-int compress_device(compams_context* c, const float* grads) {
+int compress_device(compams_context* c, const void* grads) {
     ++c->steps_done;
     if (c->compressor == COMPAMS_BLOCKSIGN) {
         c->scales_cur ^= 1;
@@ -359,7 +359,7 @@ int apply_device(compams_context* c, float* theta) {
     return COMPAMS_OK;
 }
 
-int step_device(compams_context* c, const float* grads, float* theta) {
+int step_device(compams_context* c, const void* grads, float* theta) {
     if (c->compressor == COMPAMS_TOPK && c->identity) {
         ++c->steps_done;
         return run_kernel(c, COMPAMS_K_DENSE_MEAN_AMSGRAD, [&] { return launch_dense_mean_amsgrad(c, grads, theta); });
@@ -430,15 +430,19 @@ int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total
                          beta2, eps);
 }
 
-int compams_compress(compams_handle c, const float* grads) {
-    if (!c || !grads || (reinterpret_cast<uintptr_t>(grads) & 3u)) return COMPAMS_ERR_INVALID_ARG;
+static int compress_any(compams_handle c, const void* grads, bool bf16) {
+    if (!c || !grads || (reinterpret_cast<uintptr_t>(grads) & (bf16 ? 1u : 3u))) return COMPAMS_ERR_INVALID_ARG;
     if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;  // k = d: nothing is compressed
+    c->grad_bf16 = bf16;
     try {
         return compress_device(c, grads);
     } catch (const std::bad_alloc&) {
         return COMPAMS_ERR_ALLOC;
     }
 }
+
+int compams_compress(compams_handle c, const float* grads) { return compress_any(c, grads, false); }
+int compams_compress_bf16(compams_handle c, const void* grads_bf16) { return compress_any(c, grads_bf16, true); }
 
 int compams_apply(compams_handle c, float* theta) {
     if (!c || !theta || (reinterpret_cast<uintptr_t>(theta) & 15u)) return COMPAMS_ERR_INVALID_ARG;
@@ -450,17 +454,21 @@ int compams_apply(compams_handle c, float* theta) {
     }
 }
 
-int compams_step(compams_handle c, const float* grads, float* theta) {
+static int step_any(compams_handle c, const void* grads, float* theta, bool bf16) {
     if (!c || !grads || !theta) return COMPAMS_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(grads) & 3u) || (reinterpret_cast<uintptr_t>(theta) & 15u))
+    if ((reinterpret_cast<uintptr_t>(grads) & (bf16 ? 1u : 3u)) || (reinterpret_cast<uintptr_t>(theta) & 15u))
         return COMPAMS_ERR_INVALID_ARG;
     if (c->n != c->n_total) return COMPAMS_ERR_INVALID_ARG;  // the other workers' messages have to be exchanged first
+    c->grad_bf16 = bf16;
     try {
         return step_device(c, grads, theta);
     } catch (const std::bad_alloc&) {
         return COMPAMS_ERR_ALLOC;
     }
 }
+
+int compams_step(compams_handle c, const float* grads, float* theta) { return step_any(c, grads, theta, false); }
+int compams_step_bf16(compams_handle c, const void* grads_bf16, float* theta) { return step_any(c, grads_bf16, theta, true); }
 
 int compams_step_host(compams_handle c, const float* grads_host, float* theta_host) {
     if (!c || !grads_host || !theta_host || c->n != c->n_total) return COMPAMS_ERR_INVALID_ARG;
@@ -483,6 +491,7 @@ int compams_step_host(compams_handle c, const float* grads_host, float* theta_ho
     CU(cudaMemcpyAsync(c->stage_grads, grads_host, gbytes, cudaMemcpyHostToDevice, c->stream));
     CU(cudaMemcpyAsync(c->stage_theta, theta_host, tbytes, cudaMemcpyHostToDevice, c->stream));
     int rc;
+    c->grad_bf16 = false;
     try {
         rc = step_device(c, c->stage_grads, c->stage_theta);
     } catch (const std::bad_alloc&) {

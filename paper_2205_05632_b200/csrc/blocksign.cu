@@ -35,16 +35,17 @@ __device__ __forceinline__ double abs_as_double(float x) {
 
 // One warp's 1024 consecutive coordinates starting at rw (relative to the block; rw may be negative
 // or reach past the block in a tile at either end of it: such coordinates are skipped).
-template <bool FULL>
-__device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int rw,
+template <bool FULL, typename GT>
+__device__ __forceinline__ void bs_sweep_tile(const GT* __restrict__ g, float* __restrict__ e, int len, int rw,
                                               int lane, bool deferred, float sp, double& acc, uint32_t& mymask) {
     const int cg = align_class(g + rw), ce = align_class(e + rw);
+    constexpr int NB = 2;  // iterations whose loads are in flight together
 #pragma unroll
-    for (int bt = 0; bt < kIters / 2; ++bt) {
-        float4 gv[2], ev[2];
+    for (int bt = 0; bt < kIters / NB; ++bt) {
+        float4 gv[NB], ev[NB];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int r = rw + (bt * 2 + u) * 128 + lane * 4;
+        for (int u = 0; u < NB; ++u) {
+            const int r = rw + (bt * NB + u) * 128 + lane * 4;
             if (FULL || (r >= 0 && r + 3 < len)) {
                 gv[u] = load4_stream(g + r, cg);
                 ev[u] = load4(e + r, ce);
@@ -53,7 +54,7 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const bool live = (unsigned)(r + k) < (unsigned)len;
-                    gt[k] = live ? __ldg(g + r + k) : 0.0f;
+                    gt[k] = live ? load1_stream(g + r + k) : 0.0f;
                     et[k] = live ? e[r + k] : 0.0f;
                 }
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
@@ -61,8 +62,8 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
             }
         }
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int it = bt * 2 + u;
+        for (int u = 0; u < NB; ++u) {
+            const int it = bt * NB + u;
             const int r = rw + it * 128 + lane * 4;
             float xs[4];
             uint32_t nib = 0;
@@ -99,7 +100,8 @@ __device__ __forceinline__ void bs_sweep_tile(const float* __restrict__ g, float
 // sign words stay indexed by coordinate: word q of the block takes its low 32 - s bits from the
 // q-th group of 32 shifted coordinates and its high s bits from the next group. The word a tile
 // shares with the next tile is put together by bs_scales from the two shares left in `edge`.
-__global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffers b, const float* __restrict__ G,
+template <typename GT>
+__global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffers b, const GT* __restrict__ G,
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     __shared__ uint32_t sh_first[kWarps];
@@ -111,7 +113,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffe
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row0 = (int64_t)i * t.d + ti.o;
     const int s = (int)(row0 & 31);
-    const float* g = G + row0;
+    const GT* g = G + row0;
     float* e = b.E + row0;
     const float sp = deferred ? b.scales_prev[(size_t)i * t.M + blk] : 0.0f;
     const int r0s = ti.r0 - s;
@@ -291,9 +293,14 @@ static BsBuffers own_rows(const compams_context* c) {
     return b;
 }
 
-cudaError_t launch_bs_sweep(compams_context* c, const float* grads) {
+cudaError_t launch_bs_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    bs_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), grads, c->e_is_x ? 1 : 0, c->segp);
+    if (c->grad_bf16)
+        bs_sweep_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads,
+                                                                     c->e_is_x ? 1 : 0, c->segp);
+    else
+        bs_sweep_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const float*)grads,
+                                                                 c->e_is_x ? 1 : 0, c->segp);
     return cudaGetLastError();
 }
 

@@ -100,6 +100,32 @@ __device__ __forceinline__ float4 load4_stream(const float* p, int cls) {
     return r;
 }
 
+// Gradients may also arrive as bfloat16, passed as their 16-bit patterns: widening to fp32 is exact
+// (the pattern shifted left by 16), so x = g + e is the same fp32 addition as with fp32 gradients
+// of those values. The class of a bfloat16 pointer is its address in elements modulo 4: class 0
+// allows one 64-bit access for 4 elements, class 2 two 32-bit ones, odd classes four 16-bit ones.
+typedef uint16_t bf16_bits;
+__device__ __forceinline__ int align_class(const bf16_bits* p) { return (int)((reinterpret_cast<uintptr_t>(p) >> 1) & 3u); }
+__device__ __forceinline__ float widen(bf16_bits h) { return __uint_as_float((uint32_t)h << 16); }
+__device__ __forceinline__ float load1_stream(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float load1_stream(const bf16_bits* p) { return widen(__ldg(p)); }
+__device__ __forceinline__ float4 load4_stream(const bf16_bits* p, int cls) {
+    uint32_t lo, hi;
+    if (cls == 0) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+        lo = v.x;
+        hi = v.y;
+    } else if (cls == 2) {
+        lo = __ldg(reinterpret_cast<const uint32_t*>(p));
+        hi = __ldg(reinterpret_cast<const uint32_t*>(p + 2));
+    } else {
+        lo = (uint32_t)__ldg(p) | ((uint32_t)__ldg(p + 1) << 16);
+        hi = (uint32_t)__ldg(p + 2) | ((uint32_t)__ldg(p + 3) << 16);
+    }
+    return make_float4(__uint_as_float(lo << 16), __uint_as_float(lo & 0xffff0000u), __uint_as_float(hi << 16),
+                       __uint_as_float(hi & 0xffff0000u));
+}
+
 // Plain (cached) load of 4 consecutive floats.
 __device__ __forceinline__ float4 load4(const float* p, int cls) {
     float4 r;

@@ -110,6 +110,7 @@ struct compams_context {
     int32_t n_total = 0;  // workers the server averages over (> n when the workers are sharded over several handles)
     int32_t row0 = 0;     // index of this handle's first worker among the n_total
     int64_t d = 0;
+    bool grad_bf16 = false;  // the gradients of the call being enqueued are bfloat16 (16-bit patterns), not fp32
     int32_t M = 0;
     int32_t compressor = 0;
     double k_ratio = 1.0;
@@ -166,13 +167,13 @@ struct compams_context {
 namespace compams {
 
 // Each launcher enqueues one kernel on ctx->stream and returns the launch status.
-cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, float* theta);
-cudaError_t launch_bs_sweep(compams_context* c, const float* grads);
+cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, float* theta);
+cudaError_t launch_bs_sweep(compams_context* c, const void* grads);
 cudaError_t launch_bs_scales(compams_context* c);
 cudaError_t launch_bs_apply(compams_context* c, float* theta);
 cudaError_t launch_bs_materialize(compams_context* c);
-cudaError_t launch_topk_small(compams_context* c, const float* grads);
-cudaError_t launch_topk_sweep(compams_context* c, const float* grads);
+cudaError_t launch_topk_small(compams_context* c, const void* grads);
+cudaError_t launch_topk_sweep(compams_context* c, const void* grads);
 cudaError_t launch_topk_select(compams_context* c);
 cudaError_t launch_topk_dense(compams_context* c);
 cudaError_t launch_topk_materialize(compams_context* c);

@@ -12,7 +12,8 @@
 namespace compams {
 
 // One CTA per 1024 coordinates: one float4 group per thread, the workers' rows read one after another.
-__global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const float* __restrict__ G,
+template <typename GT>
+__global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const GT* __restrict__ G,
                                                                          float* __restrict__ gbar, float* __restrict__ m,
                                                                          float* __restrict__ v, float* __restrict__ vhat,
                                                                          float* __restrict__ theta, HyperParams hp) {
@@ -21,10 +22,10 @@ __global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t
     if (q < groups) {
         const int64_t j = q << 2;
         double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-        const float* p = G + j;
+        const GT* p = G + j;
 #pragma unroll 4
         for (int32_t i = 0; i < n; ++i) {
-            const float* pi = p + (size_t)i * (size_t)d;
+            const GT* pi = p + (size_t)i * (size_t)d;
             float4 g = load4_stream(pi, align_class(pi));
             a0 += (double)g.x;
             a1 += (double)g.y;
@@ -51,7 +52,7 @@ __global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t
     if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
         const int64_t j = (groups << 2) + threadIdx.x;
         double a = 0.0;
-        for (int32_t i = 0; i < n; ++i) a += (double)G[(size_t)i * (size_t)d + (size_t)j];
+        for (int32_t i = 0; i < n; ++i) a += (double)load1_stream(G + (size_t)i * (size_t)d + (size_t)j);
         float gb = mean_from_acc(a, hp);
         float mm = m[j], vv = v[j], vh = vhat[j], th = theta[j];
         amsgrad_update(gb, mm, vv, vh, th, hp);
@@ -148,12 +149,16 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
     }
 }
 
-cudaError_t launch_dense_mean_amsgrad(compams_context* c, const float* grads, float* theta) {
+cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, float* theta) {
     int64_t groups = c->d >> 2;
     int grid = (int)((groups + kThreads - 1) / kThreads);
     if (grid < 1) grid = 1;
-    dense_mean_amsgrad_kernel<<<grid, kThreads, 0, c->stream>>>(c->n, c->d, grads, c->gbar, c->m, c->v, c->vhat, theta,
-                                                                c->hp);
+    if (c->grad_bf16)
+        dense_mean_amsgrad_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, (const bf16_bits*)grads, c->gbar,
+                                                                               c->m, c->v, c->vhat, theta, c->hp);
+    else
+        dense_mean_amsgrad_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, (const float*)grads, c->gbar, c->m,
+                                                                           c->v, c->vhat, theta, c->hp);
     return cudaGetLastError();
 }
 

@@ -77,8 +77,8 @@ __device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int len
 // boundary shifted down to a 128-byte line of G and E: r0 may be negative and the tile may reach
 // past the block; such coordinates are skipped. `row0` is the index of the block's first element
 // in E ([n, d] flattened), which is also its bit in the kept map; row0 + r0 is a multiple of 32.
-template <bool FULL>
-__device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, float* __restrict__ e, int len, int r0,
+template <bool FULL, typename GT>
+__device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float* __restrict__ e, int len, int r0,
                                                 int warp, int lane, uint32_t tau_hat, uint32_t coord0, int64_t row0,
                                                 uint2* sh_cand, uint32_t* sh_cnt, uint32_t* g_cnt, uint2* g_out,
                                                 uint32_t cap, const uint32_t* __restrict__ kept, int64_t map_words) {
@@ -90,12 +90,13 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
         const int64_t w = ((row0 + lane_r(r0, warp, 0, 0)) >> 5) + lane;
         mapw = w < map_words ? __ldg(kept + w) : 0u;
     }
+    constexpr int NB = 2;  // iterations whose loads are in flight together
 #pragma unroll
-    for (int bt = 0; bt < kIters / 2; ++bt) {
-        float4 gv[2], ev[2];
+    for (int bt = 0; bt < kIters / NB; ++bt) {
+        float4 gv[NB], ev[NB];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int r = lane_r(r0, warp, bt * 2 + u, lane);
+        for (int u = 0; u < NB; ++u) {
+            const int r = lane_r(r0, warp, bt * NB + u, lane);
             if (FULL || (r >= 0 && r + 3 < len)) {
                 gv[u] = load4_stream(g + r, cg_);
                 ev[u] = load4(e + r, ce);
@@ -104,7 +105,7 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const bool live = (unsigned)(r + k) < (unsigned)len;
-                    gt[k] = live ? __ldg(g + r + k) : 0.0f;
+                    gt[k] = live ? load1_stream(g + r + k) : 0.0f;
                     et[k] = live ? e[r + k] : 0.0f;
                 }
                 gv[u] = make_float4(gt[0], gt[1], gt[2], gt[3]);
@@ -112,12 +113,12 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
             }
         }
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int r = lane_r(r0, warp, bt * 2 + u, lane);
+        for (int u = 0; u < NB; ++u) {
+            const int r = lane_r(r0, warp, bt * NB + u, lane);
             // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, line 8).
             // Placed after the batch's loads have been issued: the shuffle waits for the map word.
             const uint32_t kb4 =
-                (__shfl_sync(0xffffffffu, mapw, (bt * 2 + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
+                (__shfl_sync(0xffffffffu, mapw, (bt * NB + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
             float xs[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -148,7 +149,8 @@ __device__ __forceinline__ void topk_sweep_tile(const float* __restrict__ g, flo
 // Tiles are shifted down by (i d + o) mod 32, the position of the block's first element within a
 // 128-byte line of G and E, so that every warp access covers whole lines (with rows that start
 // mid-line a warp's 512 bytes straddle five lines instead of four: measured 7 % slower).
-__global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const float* __restrict__ G,
+template <typename GT>
+__global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
                                                                  const __grid_constant__ SegParams sp_) {
     __shared__ uint2 sh_cand[kTileCand];
     __shared__ uint32_t sh_cnt, sh_base;
@@ -164,7 +166,7 @@ __global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkB
     if (threadIdx.x == 0) sh_cnt = 0u;
     __syncthreads();
     const int64_t row0 = (int64_t)i * t.d + ti.o;
-    const float* g = G + row0;
+    const GT* g = G + row0;
     float* e = b.E + row0;
     const int r0s = ti.r0 - (int)(row0 & 31);
     if (r0s >= 0 && r0s + kTile <= ti.len)
@@ -1060,7 +1062,8 @@ __global__ void __launch_bounds__(kThreads) topk_dense_kernel(Tables t, TopkBuff
 // ------------------------------------------------------------------------------------------
 // small blocks: the whole selection inside one CTA's shared memory
 
-__global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuffers b, const float* __restrict__ G) {
+template <typename GT>
+__global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G) {
     __shared__ uint32_t xs[kSmallMax];
     __shared__ uint32_t hist[256];
     __shared__ uint32_t scratch[kWarps];
@@ -1070,9 +1073,9 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
     const int64_t o = t.off[blk];
     const int len = (int)(t.off[blk + 1] - o);
     const uint32_t kb = (uint32_t)(b.seg_off[blk + 1] - b.seg_off[blk]);
-    const float* g = G + (size_t)i * (size_t)t.d + (size_t)o;
+    const GT* g = G + (size_t)i * (size_t)t.d + (size_t)o;
     float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
-    for (int r = threadIdx.x; r < len; r += kThreads) xs[r] = __float_as_uint(__fadd_rn(__ldg(g + r), e[r]));
+    for (int r = threadIdx.x; r < len; r += kThreads) xs[r] = __float_as_uint(__fadd_rn(load1_stream(g + r), e[r]));
 
     // radix select over the 31-bit key: digits of 8, 8, 8 and 7 bits from the top
     uint32_t prefix = 0, k_rem = kb;
@@ -1229,15 +1232,22 @@ static TopkBuffers own_rows(const compams_context* c) {
     return b;
 }
 
-cudaError_t launch_topk_small(compams_context* c, const float* grads) {
+cudaError_t launch_topk_small(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tk.nsmall, (unsigned)c->n);
-    topk_small_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), grads);
+    if (c->grad_bf16)
+        topk_small_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads);
+    else
+        topk_small_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const float*)grads);
     return cudaGetLastError();
 }
 
-cudaError_t launch_topk_sweep(compams_context* c, const float* grads) {
+cudaError_t launch_topk_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    topk_sweep_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), grads, c->segp);
+    if (c->grad_bf16)
+        topk_sweep_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads,
+                                                                       c->segp);
+    else
+        topk_sweep_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const float*)grads, c->segp);
     return cudaGetLastError();
 }
 

@@ -80,7 +80,8 @@ class Pair:
         s = self.step_no
         Gd = G.to("cuda")
         self.gpu.step(Gd, self.theta_gpu)
-        self.cpu.step(np.ascontiguousarray(G.detach().cpu().numpy()), self.theta_cpu)
+        # bfloat16 gradients: the oracle is fed the fp32 numbers with the same values (widening is exact)
+        self.cpu.step(np.ascontiguousarray(G.detach().float().cpu().numpy()), self.theta_cpu)
         assert self.gpu.check_status() == 0
         cnt = self.inexact
         if self.compressor == TOPK and not self.identity:

@@ -26,6 +26,10 @@ def _randn(n, d):
     return lambda gen, t: torch.randn(n, d, generator=gen, device="cuda")
 
 
+def _randn_bf16(n, d):
+    return lambda gen, t: torch.randn(n, d, generator=gen, device="cuda").bfloat16()
+
+
 # ------------------------------------------------------------------ mid-size cases: several tiles, ragged tails
 
 RAGGED = [0, 10, 74, 1098, 5194, 5195, 13387 + 5, 13392 + 3 * 8192 + 1234, 13392 + 3 * 8192 + 1234 + 4097]
@@ -49,6 +53,37 @@ def test_blocksign_ragged_blocks(n, check_e_every):
 @pytest.mark.parametrize("comp", [TOPK, BLOCKSIGN])
 def test_single_block_sizes_around_tile_edges(d, comp):
     _pair_run(2, d, [0, d], comp, 0.1, _randn(2, d), steps=3)
+
+
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (TOPK, 0.3), (TOPK, 1.0), (BLOCKSIGN, 1.0)])
+@pytest.mark.parametrize("n", [1, 3, 4])
+def test_bfloat16_gradients_ragged_blocks(comp, ratio, n):
+    # d = 3 mod 4 and odd block offsets: rows and blocks of the bfloat16 tensor start in every alignment class
+    d = RAGGED[-1]
+    assert d % 4 == 3
+    _pair_run(n, d, RAGGED, comp, ratio, _randn_bf16(n, d))
+
+
+def test_bfloat16_and_fp32_gradients_may_alternate():
+    d = 3 * 8192 + 77
+    mixed = lambda gen, t: (torch.randn(2, d, generator=gen, device="cuda").bfloat16() if t % 2 else
+                            torch.randn(2, d, generator=gen, device="cuda"))
+    for comp in (TOPK, BLOCKSIGN):
+        _pair_run(2, d, [0, d], comp, 0.02, mixed, steps=5)
+
+
+def test_bfloat16_gradients_resnet18_shapes_blocksign_and_topk():
+    w = W.config2("cuda")
+    theta = w.start()
+    from parity import Pair
+    for comp, ratio, offs in ((BLOCKSIGN, 1.0, w.block_offsets), (TOPK, 0.01, np.array([0, w.d]))):
+        p = Pair(4, w.d, offs, comp, ratio)
+        try:
+            p.start(theta)
+            for t in range(3):
+                p.step(w.grads()[:4].contiguous().bfloat16(), check_e=(t == 2))
+        finally:
+            p.close()
 
 
 def test_rows_not_multiple_of_four_use_all_alignment_classes():
