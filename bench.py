@@ -53,9 +53,9 @@ def measured_peak_gbs():
 # profiles/dram_traffic_bench_resnet18_n16.md, with a hash of the kernel's source at the time of the
 # capture: once the source changes the figure no longer describes the kernel and None is reported.
 TRAFFIC = {
-    "bs_sweep": (2118436352, "blocksign.cu", "f3a7b7012a23355f"),
-    "topk_sweep": (2163855104, "topk.cu", "0bfb0dcf8c109638"),
-    "dense_mean_amsgrad": (1098390784, "dense.cu", "e38cb066468e3d5e"),
+    "bs_sweep": (2120694784, "blocksign.cu", "74720844c02bea8d"),
+    "topk_sweep": (2163284224, "topk.cu", "995e76e14a8d06e0"),
+    "dense_mean_amsgrad": (1100273664, "dense.cu", "4831161e6e70d773"),
 }
 
 
