@@ -24,7 +24,7 @@ constexpr int kSurvCapBig = 65536;       // threshold-bin candidates of a long l
 constexpr int kSurvSmem = 4096;          // ... of which this many fit the finishing CTA's shared memory
 constexpr int kRankMax = 256;            // ... and up to this many are ranked pair by pair
 constexpr int kSelBins = 4096;           // bins of the candidate select's first histogram
-constexpr int kSelectSingleMax = 24576;  // candidate capacity up to which one CTA handles a segment
+constexpr int kSelectSingleMax = 98304;  // candidate capacity up to which one CTA handles a segment
 
 // Per (worker, large block) Top-k selection state.
 struct SegState {
