@@ -128,6 +128,17 @@ def test_blocks_of_size_one_and_tiny():
         _pair_run(3, d, offs, comp, 0.2, _randn(3, d), steps=3)
 
 
+def test_more_tiled_blocks_than_the_kernel_argument_block_list_holds():
+    # the sweeps find a tile's block in a kernel-argument copy of the block list when it has at most 168
+    # entries; beyond that they read a per-tile table in global memory
+    sizes = [4097 + 37 * (b % 23) for b in range(181)]   # Top-k: 181 tiled blocks (each above 4096 coordinates)
+    offs = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    _pair_run(2, offs[-1], offs, TOPK, 0.01, _randn(2, offs[-1]), steps=4)
+    sizes = [1 + (7 * b) % 300 for b in range(400)] + [9000, 3, 8192, 1]   # Block-Sign: every block is tiled
+    offs = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    _pair_run(3, offs[-1], offs, BLOCKSIGN, 1.0, _randn(3, offs[-1]), steps=4)
+
+
 # ------------------------------------------------------------------ degenerate inputs: ties everywhere
 
 def _quantised(n, d, levels):
