@@ -396,6 +396,7 @@ int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0,
     c->hp.omb1 = 1.0f - beta1;
     c->hp.omb2 = 1.0f - beta2;
     c->hp.eps = eps;
+    c->chain = (int64_t)n * d <= kChainMaxElems;
     c->hp.nf = (float)n_total;
     c->hp.inv_nf = ((n_total & (n_total - 1)) == 0) ? 1.0f / (float)n_total : 0.0f;
     int rc;

@@ -9,6 +9,10 @@
 #include "../../include/compams.h"
 #include "common.cuh"
 
+#ifndef COMPAMS_CHAIN_MAX
+#define COMPAMS_CHAIN_MAX ((int64_t)1 << 25)
+#endif
+
 namespace compams {
 
 constexpr int kSmallMax = 4096;    // Top-k blocks up to this size are selected inside one CTA's shared memory
@@ -24,6 +28,7 @@ constexpr int kSurvCapBig = 65536;       // threshold-bin candidates of a long l
 constexpr int kSurvSmem = 4096;          // ... of which this many fit the finishing CTA's shared memory
 constexpr int kRankMax = 256;            // ... and up to this many are ranked pair by pair
 constexpr int kSelBins = 4096;           // bins of the candidate select's first histogram
+constexpr int64_t kChainMaxElems = COMPAMS_CHAIN_MAX;  // n d up to which a step's kernels are chained
 constexpr int kSelectSingleMax = 98304;  // candidate capacity up to which one CTA handles a segment
 
 // Per (worker, large block) Top-k selection state.
@@ -110,6 +115,7 @@ struct compams_context {
     int32_t n_total = 0;  // workers the server averages over (> n when the workers are sharded over several handles)
     int32_t row0 = 0;     // index of this handle's first worker among the n_total
     int64_t d = 0;
+    bool chain = false;      // small problem: the Top-k kernels of a step are launched as programmatic dependents
     bool grad_bf16 = false;  // the gradients of the call being enqueued are bfloat16 (16-bit patterns), not fp32
     int32_t M = 0;
     int32_t compressor = 0;

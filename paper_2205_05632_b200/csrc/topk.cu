@@ -152,6 +152,8 @@ __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float*
 template <typename GT>
 __global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
                                                                  const __grid_constant__ SegParams sp_) {
+    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint2 sh_cand[kTileCand];
     __shared__ uint32_t sh_cnt, sh_base;
     const TileInfo ti = sp_.nseg ? find_tile(sp_, blockIdx.x) : load_tile(t.tiles, blockIdx.x);
@@ -269,6 +271,8 @@ __device__ __forceinline__ uint32_t offset_digit(uint32_t xbits, uint32_t tau_ha
 
 __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                int nlist) {
+    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint32_t local[kSelBins];  // histogram of the list
     __shared__ uint2 surv[kSurvCap];
     __shared__ uint32_t scratch[kSelWarps];
@@ -468,6 +472,8 @@ __global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, Topk
 
 __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                 int nlist, int parts) {
+    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint32_t local[kSelBins];
     __shared__ uint32_t scratch[kWarps];
     __shared__ uint32_t sh_bin[3], sh_edge[3];
@@ -564,6 +570,8 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
 
 __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                 int nlist, int parts) {
+    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint2 surv[kSurvSmem];
     __shared__ uint32_t sh_hist[kThreads];
     __shared__ uint32_t scratch[kWarps];
@@ -1156,6 +1164,7 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 // The same walk zeroes e at the kept coordinates (they were left holding x by the sweep).
 
 __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count, int32_t row0) {
+    dependency_wait();
     allow_dependents();
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     // the first n * nseg threads also close the step for one large-block segment each: exactly k_b
@@ -1243,6 +1252,13 @@ cudaError_t launch_topk_small(compams_context* c, const void* grads) {
 
 cudaError_t launch_topk_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
+    if (c->chain) {
+        if (c->grad_bf16)
+            return launch_after(topk_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                                (const bf16_bits*)grads, c->segp);
+        return launch_after(topk_sweep_kernel<float>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                            (const float*)grads, c->segp);
+    }
     if (c->grad_bf16)
         topk_sweep_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads,
                                                                        c->segp);
@@ -1251,21 +1267,29 @@ cudaError_t launch_topk_sweep(compams_context* c, const void* grads) {
     return cudaGetLastError();
 }
 
+// On small problems the kernels of a step are launched as programmatic dependents of one another (each
+// waits for its predecessor before its first global access): the launch latency and the prologue of a
+// kernel then overlap the tail of the one before, which is most of what such a step costs.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_chained(const compams_context* c, void (*kernel)(KArgs...), dim3 grid, dim3 block, Args... args) {
+    if (c->chain) return launch_after(kernel, grid, block, c->stream, args...);
+    kernel<<<grid, block, 0, c->stream>>>(static_cast<KArgs>(args)...);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_topk_select(compams_context* c) {
     cudaError_t e = cudaSuccess;
     const TopkBuffers b = own_rows(c);
-    if (c->n_sel_small > 0) {
-        topk_select_kernel<<<(unsigned)((int64_t)c->n * c->n_sel_small), kSelThreads, 0, c->stream>>>(
-            c->tab, b, c->sel_small, c->n_sel_small);
-        e = cudaGetLastError();
-    }
+    if (c->n_sel_small > 0)
+        e = launch_chained(c, topk_select_kernel, dim3((unsigned)((int64_t)c->n * c->n_sel_small)), dim3(kSelThreads),
+                           c->tab, b, (const int32_t*)c->sel_small, c->n_sel_small);
     if (e != cudaSuccess || c->n_sel_big == 0) return e;
-    const unsigned grid = (unsigned)((int64_t)c->n * c->n_sel_big * c->sel_parts);
-    topk_selhist_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, c->sel_big, c->n_sel_big, c->sel_parts);
-    e = cudaGetLastError();
+    const dim3 grid((unsigned)((int64_t)c->n * c->n_sel_big * c->sel_parts));
+    e = launch_chained(c, topk_selhist_kernel, grid, dim3(kThreads), c->tab, b, (const int32_t*)c->sel_big, c->n_sel_big,
+                       c->sel_parts);
     if (e != cudaSuccess) return e;
-    topk_selemit_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, b, c->sel_big, c->n_sel_big, c->sel_parts);
-    return cudaGetLastError();
+    return launch_chained(c, topk_selemit_kernel, grid, dim3(kThreads), c->tab, b, (const int32_t*)c->sel_big,
+                          c->n_sel_big, c->sel_parts);
 }
 
 cudaError_t launch_topk_dense(compams_context* c) {
@@ -1293,6 +1317,9 @@ cudaError_t launch_topk_scatter(compams_context* c) {
     // one thread per message entry of every worker (>= n * nseg: every block keeps at least one entry)
     const int64_t count = (int64_t)c->n_total * c->K;
     const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
+    // (a sharded handle's exchange sits in front of this kernel: a plain launch waits for it)
+    if (c->chain && c->n == c->n_total)
+        return launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count, c->row0);
     topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, c->row0);
     return cudaGetLastError();
 }
