@@ -39,10 +39,14 @@ template <bool FULL, typename GT>
 __device__ __forceinline__ void bs_sweep_tile(const GT* __restrict__ g, float* __restrict__ e, int len, int rw,
                                               int lane, bool deferred, float sp, double& acc, uint32_t& mymask) {
     const int cg = align_class(g + rw), ce = align_class(e + rw);
-    constexpr int NB = 2;  // iterations whose loads are in flight together
-#pragma unroll
-    for (int bt = 0; bt < kIters / NB; ++bt) {
-        float4 gv[NB], ev[NB];
+    // One iteration (4 coordinates per lane) is worked on while the next one's loads are already in flight
+    // (two register buffers that alternate; the loop is fully unrolled). Small batches keep the kernel at
+    // 32 registers, eight CTAs per SM: measured 0.329 ms against 0.355 ms for two-iteration batches without
+    // prefetch at five CTAs per SM (ResNet-18 shapes, n = 16), the rate of a plain device copy.
+    constexpr int NB = 1;
+    constexpr int NBT = kIters / NB;
+    float4 gbuf[2][NB], ebuf[2][NB];
+    auto load_batch = [&](int bt, float4 (&gv)[NB], float4 (&ev)[NB]) {
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
             const int r = rw + (bt * NB + u) * 128 + lane * 4;
@@ -61,6 +65,13 @@ __device__ __forceinline__ void bs_sweep_tile(const GT* __restrict__ g, float* _
                 ev[u] = make_float4(et[0], et[1], et[2], et[3]);
             }
         }
+    };
+    load_batch(0, gbuf[0], ebuf[0]);
+#pragma unroll
+    for (int bt = 0; bt < NBT; ++bt) {
+        float4 (&gv)[NB] = gbuf[bt & 1];
+        float4 (&ev)[NB] = ebuf[bt & 1];
+        if (bt + 1 < NBT) load_batch(bt + 1, gbuf[(bt + 1) & 1], ebuf[(bt + 1) & 1]);
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
             const int it = bt * NB + u;
@@ -101,7 +112,7 @@ __device__ __forceinline__ void bs_sweep_tile(const GT* __restrict__ g, float* _
 // q-th group of 32 shifted coordinates and its high s bits from the next group. The word a tile
 // shares with the next tile is put together by bs_scales from the two shares left in `edge`.
 template <typename GT>
-__global__ void __launch_bounds__(kThreads, 5) bs_sweep_kernel(Tables t, BsBuffers b, const GT* __restrict__ G,
+__global__ void __launch_bounds__(kThreads, 8) bs_sweep_kernel(Tables t, BsBuffers b, const GT* __restrict__ G,
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     __shared__ uint32_t sh_first[kWarps];

@@ -12,8 +12,10 @@
 namespace compams {
 
 // One CTA per 1024 coordinates: one float4 group per thread, the workers' rows read one after another.
+// Eight CTAs per SM (32 registers, a few spilled words) beat six (40 registers): 0.187 against 0.200 ms on
+// ResNet-18 shapes, n = 16; requesting the optimizer state ahead of the rows costs registers and is slower.
 template <typename GT>
-__global__ void __launch_bounds__(kThreads, 6) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const GT* __restrict__ G,
+__global__ void __launch_bounds__(kThreads, 8) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const GT* __restrict__ G,
                                                                          float* __restrict__ gbar, float* __restrict__ m,
                                                                          float* __restrict__ v, float* __restrict__ vhat,
                                                                          float* __restrict__ theta, HyperParams hp) {

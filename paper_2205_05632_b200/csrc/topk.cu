@@ -150,7 +150,7 @@ __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float*
 // 128-byte line of G and E, so that every warp access covers whole lines (with rows that start
 // mid-line a warp's 512 bytes straddle five lines instead of four: measured 7 % slower).
 template <typename GT>
-__global__ void __launch_bounds__(kThreads, 5) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
+__global__ void __launch_bounds__(kThreads, 6) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
                                                                  const __grid_constant__ SegParams sp_) {
     dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
