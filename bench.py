@@ -53,9 +53,9 @@ def measured_peak_gbs():
 # profiles/dram_traffic_bench_resnet18_n16.md, with a hash of the kernel's source at the time of the
 # capture: once the source changes the figure no longer describes the kernel and None is reported.
 TRAFFIC = {
-    "bs_sweep": (2120694784, "blocksign.cu", "74720844c02bea8d"),
-    "topk_sweep": (2163284224, "topk.cu", "995e76e14a8d06e0"),
-    "dense_mean_amsgrad": (1100273664, "dense.cu", "4831161e6e70d773"),
+    "bs_sweep": (2117318912, "blocksign.cu", "640a88e873ea0415"),
+    "topk_sweep": (2161511424, "topk.cu", "c25ee64747557c29"),
+    "dense_mean_amsgrad": (1143972608, "dense.cu", "f68caa50395b3f5c"),
 }
 
 
