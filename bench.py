@@ -55,7 +55,7 @@ def measured_peak_gbs():
 TRAFFIC = {
     "bs_sweep": (2117154304, "blocksign.cu", "640a88e873ea0415"),
     "topk_sweep": (2162749952, "topk.cu", "f2c1237aa92a4112"),
-    "dense_mean_amsgrad": (1144125952, "dense.cu", "f68caa50395b3f5c"),
+    "dense_mean_amsgrad": (1144333312, "dense.cu", "1024694d4f0761c8"),
 }
 
 

@@ -12,10 +12,12 @@
 namespace compams {
 
 // One CTA per 1024 coordinates: one float4 group per thread, the workers' rows read one after another.
-// Eight CTAs per SM (32 registers, a few spilled words) beat six (40 registers): 0.187 against 0.200 ms on
-// ResNet-18 shapes, n = 16; requesting the optimizer state ahead of the rows costs registers and is slower.
-template <typename GT>
-__global__ void __launch_bounds__(kThreads, 8) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const GT* __restrict__ G,
+// Two builds: eight CTAs per SM (32 registers, a few spilled words) beat six (40 registers) once there are
+// rows enough to wait for - 0.187 against 0.200 ms on ResNet-18 shapes, n = 16 - and lose to them when the
+// optimizer state is most of the traffic (d = 2^26: n = 1 0.427 against 0.395 ms, n = 4 0.531 against 0.522 ms,
+// n = 8 0.677 against 0.707 ms). Requesting the state ahead of the rows costs registers and is slower.
+template <typename GT, int CTAS_PER_SM>
+__global__ void __launch_bounds__(kThreads, CTAS_PER_SM) dense_mean_amsgrad_kernel(int32_t n, int64_t d, const GT* __restrict__ G,
                                                                          float* __restrict__ gbar, float* __restrict__ m,
                                                                          float* __restrict__ v, float* __restrict__ vhat,
                                                                          float* __restrict__ theta, HyperParams hp) {
@@ -155,12 +157,24 @@ cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, flo
     int64_t groups = c->d >> 2;
     int grid = (int)((groups + kThreads - 1) / kThreads);
     if (grid < 1) grid = 1;
-    if (c->grad_bf16)
-        dense_mean_amsgrad_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, (const bf16_bits*)grads, c->gbar,
-                                                                               c->m, c->v, c->vhat, theta, c->hp);
-    else
-        dense_mean_amsgrad_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, (const float*)grads, c->gbar, c->m,
-                                                                           c->v, c->vhat, theta, c->hp);
+    const bool many_rows = c->n >= 6;
+    if (c->grad_bf16) {
+        const bf16_bits* g = (const bf16_bits*)grads;
+        if (many_rows)
+            dense_mean_amsgrad_kernel<bf16_bits, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+                                                                                      c->vhat, theta, c->hp);
+        else
+            dense_mean_amsgrad_kernel<bf16_bits, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+                                                                                      c->vhat, theta, c->hp);
+    } else {
+        const float* g = (const float*)grads;
+        if (many_rows)
+            dense_mean_amsgrad_kernel<float, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+                                                                                  c->vhat, theta, c->hp);
+        else
+            dense_mean_amsgrad_kernel<float, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+                                                                                  c->vhat, theta, c->hp);
+    }
     return cudaGetLastError();
 }
 
