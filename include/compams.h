@@ -5,8 +5,8 @@
  * "On Distributed Adaptive Optimization with Gradient Compression" (Li, Karimi, Li, ICLR 2022)
  * per call, with all n workers held as rows of [n, d] buffers on one GPU:
  *
- *   worker i (Algorithm 2, lines 7-8):   x_i = g_i + e_i;  g~_i = C(x_i);  e_i <- x_i - g~_i
- *   server   (Algorithm 2, lines 12-16): gbar = (1/n) sum_i g~_i;
+ *   worker i (Algorithm 2, the corrected-gradient and residual steps):   x_i = g_i + e_i;  g~_i = C(x_i);  e_i <- x_i - g~_i
+ *   server   (Algorithm 2, the server's average and update): gbar = (1/n) sum_i g~_i;
  *                                        m <- b1 m + (1-b1) gbar;  v <- b2 v + (1-b2) gbar^2;
  *                                        vhat <- max(vhat, v);  theta <- theta - lr m / sqrt(vhat + eps)
  *
@@ -53,7 +53,7 @@ enum compams_status {
 
 /* Buffers readable through compams_get_buffer. */
 enum compams_buffer {
-    COMPAMS_BUF_E = 0,            /* float  [n, d]   error accumulators e_{t+1,i} (Algorithm 2, line 8)          */
+    COMPAMS_BUF_E = 0,            /* float  [n, d]   error accumulators e_{t+1,i} (Algorithm 2, the residual update)          */
     COMPAMS_BUF_M = 1,            /* float  [d]      first moment m_t                                            */
     COMPAMS_BUF_V = 2,            /* float  [d]      second moment v_t                                           */
     COMPAMS_BUF_VHAT = 3,         /* float  [d]      running maximum vhat_t                                      */
@@ -118,7 +118,7 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
                    int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps);
 
 /*
- * compams_step - one iteration of Algorithm 2 (lines 7-8 for every worker, lines 12-16 for the
+ * compams_step - one iteration of Algorithm 2 (the corrected-gradient and residual steps for every worker, the server's average and update for the
  * server), enqueued on the handle's stream.
  *
  *   grads   device; [n, d] fp32, packed row-major (row i = g_{t,i}, row stride d), 4-byte aligned.
@@ -151,7 +151,7 @@ int compams_compress_bf16(compams_handle h, const void* grads_bf16);
 
 /*
  * compams_step_host - the same iteration for callers whose tensors live in HOST memory
- * (Algorithm 2's "send g~ to the server / receive theta" endpoints on a machine where the
+ * (the two ends of Algorithm 2's exchange with the server, on a machine where the
  * gradients are produced off-GPU).
  *
  *   grads_host  host; [n, d] fp32 packed. Copied to a device staging buffer owned by the handle.
@@ -165,8 +165,8 @@ int compams_step_host(compams_handle h, const float* grads_host, float* theta_ho
 
 /*
  * Workers sharded over several handles (several GPUs or processes), as in Algorithm 2 proper: every
- * worker compresses locally and "sends g~_{t,i} to the central server" (line 9); the server averages
- * the n compressed gradients and updates theta (lines 11-16). Here every shard also plays the server
+ * worker compresses locally and ships its compressed gradient to the server; the server averages
+ * the n compressed gradients and updates theta (the server's part). Here every shard also plays the server
  * on its own replica of theta, m, v, vhat: after the shards have exchanged their compressed gradients
  * (an all-gather of the message buffers - the only communication, and it is the caller's: this library
  * starts no collective), each applies the identical update, so the replicas stay bit-identical and
@@ -180,13 +180,13 @@ int compams_step_host(compams_handle h, const float* grads_host, float* theta_ho
  *   has no message to exchange and is refused (INVALID_ARG). compams_create(n, ...) is
  *   compams_create_sharded(n, n, 0, ...).
  *
- * compams_compress - lines 5-9 for this handle's workers: x = g + e, the compression, the residual.
+ * compams_compress - the workers' loop for this handle's workers: x = g + e, the compression, the residual.
  *   grads   device; [n_local, d] fp32 packed, 4-byte aligned; read only.
  *   Fills rows first_worker ... first_worker + n_local - 1 of the message buffers. The caller then
  *   makes the other rows hold the other shards' messages (for Block-Sign BUF_SCALES must be asked for
  *   AFTER this call: two scale buffers alternate), ordered on the handle's stream before compams_apply.
  *
- * compams_apply - lines 11-16: gbar_t = (1/n_total) sum of the n_total messages, then the AMSGrad update.
+ * compams_apply - the server's part: gbar_t = (1/n_total) sum of the n_total messages, then the AMSGrad update.
  *   theta   device; [d] fp32, 16-byte aligned; updated in place.
  *
  * compams_step on a handle with n_local == n_total is compams_compress followed by compams_apply;
@@ -213,15 +213,15 @@ int compams_set_lr(compams_handle h, float lr);
 
 /*
  * compams_get_state / compams_set_state - checkpoint and restore what Algorithm 2 carries from one
- * iteration to the next: the workers' error accumulators e_{t,i} (line 8) and the server's m_t, v_t,
- * v-hat_t (lines 13-15). theta is the caller's own tensor and the step counter does not enter the
+ * iteration to the next: the workers' error accumulators e_{t,i} (the residual update) and the server's m_t, v_t,
+ * v-hat_t (the moment and maximum updates). theta is the caller's own tensor and the step counter does not enter the
  * update (Algorithm 1 has no bias correction), so these four are the whole state.
  *
  *   e         DEVICE, [n, d] packed rows, or null to skip. With k_b = d_b in every block the
  *             accumulators are identically zero and not stored: get writes zeros, set ignores e.
  *   m, v, vhat  DEVICE, [d] each, or null to skip.
  *
- * get copies out the values line 8 defines (a residual still to be finished is finished first);
+ * get copies out the values the residual update defines (a residual still to be finished is finished first);
  * set copies in and forgets what the library had derived from earlier steps (threshold
  * predictions), which changes the path a selection takes, never its result. Both run on the
  * handle's stream, asynchronously; the caller's buffers must stay valid until that work is done.
@@ -240,7 +240,7 @@ int compams_set_state(compams_handle h, const float* e, const float* m, const fl
  *             bit per coordinate plus 32 bits per block scale (Block-Sign); equal to [0] when
  *             every block keeps all its coordinates;
  *         [2] the 32-bit coordinate indices that accompany Top-k values (0 otherwise). The
- *             paper's "around 100x" for Top-0.01 is [0] / [1]; a wire format also pays [2].
+ *             roughly hundredfold saving the paper reports for Top-0.01 is [0] / [1]; a wire format also pays [2].
  */
 int compams_bits_transmitted(compams_handle h, uint64_t* out);
 
@@ -254,7 +254,7 @@ int compams_bits_transmitted(compams_handle h, uint64_t* out);
  *
  * The contents are those of the last enqueued step once the stream has reached that point;
  * they stay valid until the next compams_step / compams_destroy. Asking for BUF_E enqueues
- * one extra kernel that finishes line 8 of Algorithm 2 in place: the step itself leaves the
+ * one extra kernel that finishes the residual update of Algorithm 2 in place: the step itself leaves the
  * corrected gradient x in E (Block-Sign: all of it; Top-k: at the kept coordinates, which are
  * recorded in a bit map) and applies e = x - g~ when E is next read, by the next iteration's sweep
  * or by this call; the values are identical either way.
@@ -298,8 +298,8 @@ int64_t compams_launch_count(compams_handle h);
  * library's device image, held by every GPU that loads the library until the process exits.
  *
  * What it computes, for every worker i over ONE block covering all d coordinates: the corrected
- * gradient x_i = g_i + e_i (Algorithm 2, line 7), written over x_state; the sign bit of every x_ij;
- * and the scale ||x_i||_1 / d (Definition 2). The residual of line 8 is deferred exactly as in
+ * gradient x_i = g_i + e_i (Algorithm 2, the corrected-gradient step), written over x_state; the sign bit of every x_ij;
+ * and the scale ||x_i||_1 / d (Definition 2). The residual update is deferred exactly as in
  * compams_step: with deferred != 0, x_state holds the PREVIOUS call's x and scales_prev that call's
  * scales, and e_i = x_prev - sign(x_prev) * scale_prev is formed on the fly; with deferred == 0,
  * x_state holds e itself (all zeros before the first step) and scales_prev is not read.

@@ -246,7 +246,7 @@ class CompAMS:
                "compams_step")
 
     def compress(self, grads: torch.Tensor) -> None:
-        """Worker side of one iteration (Algorithm 2, lines 5-9) for this optimizer's workers."""
+        """Worker side of one iteration (Algorithm 2, the workers' loop) for this optimizer's workers."""
         if not (grads.is_cuda and grads.dtype in (torch.float32, torch.bfloat16) and grads.is_contiguous()
                 and tuple(grads.shape) == (self.n, self.d)):
             raise CompAMSError("grads must be a contiguous float32 or bfloat16 CUDA tensor of shape [n, d]")
@@ -254,7 +254,7 @@ class CompAMS:
         _check(fn(self._h, ctypes.c_void_p(grads.data_ptr())), "compams_compress")
 
     def apply(self, theta: torch.Tensor) -> None:
-        """Server side (lines 11-16) over the messages of all n_total workers."""
+        """Server side (the server's part) over the messages of all n_total workers."""
         if not (theta.is_cuda and theta.dtype == torch.float32 and theta.is_contiguous()
                 and tuple(theta.shape) == (self.d,)):
             raise CompAMSError("theta must be a contiguous float32 CUDA tensor of shape [d]")

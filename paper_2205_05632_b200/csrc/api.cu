@@ -322,7 +322,7 @@ int run_kernel(compams_context* c, int kernel, F&& launch) {
     return COMPAMS_OK;
 }
 
-// Worker side of one iteration (Algorithm 2, lines 5-9) for this handle's workers: x = g + e, the
+// Worker side of one iteration (Algorithm 2, the workers' loop) for this handle's workers: x = g + e, the
 // compression, the residual; the compressed gradients land in this handle's rows of the message buffers.
 int compress_device(compams_context* c, const void* grads) {
     ++c->steps_done;
@@ -348,7 +348,7 @@ int compress_device(compams_context* c, const void* grads) {
     return COMPAMS_OK;
 }
 
-// Server side (Algorithm 2, lines 11-16): average of the n_total compressed gradients and AMSGrad.
+// Server side (Algorithm 2, the server's part): average of the n_total compressed gradients and AMSGrad.
 int apply_device(compams_context* c, float* theta) {
     if (c->compressor == COMPAMS_BLOCKSIGN) {
         return run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); });
@@ -523,7 +523,7 @@ int compams_set_lr(compams_handle c, float lr) {
     return COMPAMS_OK;
 }
 
-// Finishes line 8 where it has been deferred, so that E holds e.
+// Finishes the residual update where it has been deferred, so that E holds e.
 static int finish_residual(compams_context* c) {
     if (c->compressor == COMPAMS_TOPK && !c->identity && c->e_mask_pending) {
         RC(run_kernel(c, COMPAMS_K_TOPK_MATERIALIZE, [&] { return launch_topk_materialize(c); }));

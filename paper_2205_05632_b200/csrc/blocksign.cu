@@ -1,17 +1,17 @@
 // Block-Sign path (Definition 2) of the COMP-AMS step.
 //
-// bs_sweep   per (worker, tile): x = g + e (Algorithm 2, line 7), x written over E, sign bits
+// bs_sweep   per (worker, tile): x = g + e (Algorithm 2, the corrected-gradient step), x written over E, sign bits
 //            packed, sum |x| of the tile in binary64.
 // bs_scales  per (worker, block): adds the tile sums in a fixed order and writes the scale
 //            ||x_B||_1 / d_B.
 // bs_apply   per coordinate: gbar = (1/n) sum_i sign(x_ij) s_{i,b} from the sign bits and
-//            scales (line 12), fused with the AMSGrad update (lines 13-16).
+//            scales (the server's average), fused with the AMSGrad update (the moment, maximum and parameter updates).
 //
-// The residual e = x - sign(x) s (line 8) needs the scale, which is known only after the whole
+// The residual e = x - sign(x) s (the residual update) needs the scale, which is known only after the whole
 // block has been read. Instead of a second pass over [n, d], E keeps x and the subtraction is
 // done when E is next read: by the next step's sweep (with the scale of the step that produced
 // x) or by bs_materialize when the caller asks for E. Both evaluate the same single fp32
-// subtraction, so the values are those of line 8 bit for bit.
+// subtraction, so the values are those of the residual update bit for bit.
 #include "context.h"
 
 namespace compams {
@@ -81,9 +81,9 @@ __device__ __forceinline__ void bs_sweep_tile(const GT* __restrict__ g, float* _
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 float xo = lane_elem(ev[u], k);
-                // deferred residual: e = x_prev - sign(x_prev) * s_prev (Algorithm 2, line 8)
+                // deferred residual: e = x_prev - sign(x_prev) * s_prev (Algorithm 2, the residual update)
                 float ee = deferred ? __fsub_rn(xo, copysignf(sp, xo)) : xo;
-                float x = __fadd_rn(lane_elem(gv[u], k), ee);  // line 7: x = g + e
+                float x = __fadd_rn(lane_elem(gv[u], k), ee);  // the corrected-gradient step: x = g + e
                 xs[k] = x;
                 const bool live = FULL || ((unsigned)(r + k) < (unsigned)len);
                 if (live) {
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kThreads) bs_scales_kernel(Tables t, BsBuffers
     if (threadIdx.x == 0) b.scales_cur[(size_t)i * t.M + blk] = __double2float_rn(S / (double)si->len);
 }
 
-// E holds x; turn it into e = x - sign(x) * s in place (Algorithm 2, line 8).
+// E holds x; turn it into e = x - sign(x) * s in place (Algorithm 2, the residual update).
 __global__ void __launch_bounds__(kThreads) bs_materialize_kernel(Tables t, float* __restrict__ E,
                                                                   const float* __restrict__ scales) {
     const int i = blockIdx.y;
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(kThreads) bs_materialize_kernel(Tables t, floa
 
 constexpr int kApplyChunk = 64;  // workers whose sign words are staged in shared memory at a time
 
-// Server side of Block-Sign (Algorithm 2, lines 12-16): one CTA per 1024 consecutive coordinates of a
+// Server side of Block-Sign (Algorithm 2, the server's average and update): one CTA per 1024 consecutive coordinates of a
 // block, one float4 group per thread. The tile's block comes from the constant bank, so the sign
 // words, the scales and the optimizer state are all requested at once. Per coordinate the sum over
 // workers of +-s_i is formed as (sum of all s_i) - 2 (sum of the s_i whose bit is set): one

@@ -55,7 +55,7 @@ struct HyperParams {
     float inv_nf;  // 1 / n when n is a power of two (then x * inv_nf == x / n bit for bit), else 0
 };
 
-// One AMSGrad coordinate update (Algorithm 2, lines 13-16). Every operation is a separately
+// One AMSGrad coordinate update (Algorithm 2, the moment, maximum and parameter updates). Every operation is a separately
 // rounded fp32 operation: no fused multiply-add, IEEE square root and division.
 __device__ __forceinline__ void amsgrad_update(float g, float& m, float& v, float& vh, float& th,
                                                const HyperParams& hp) {
@@ -65,7 +65,7 @@ __device__ __forceinline__ void amsgrad_update(float g, float& m, float& v, floa
     th = __fsub_rn(th, __fdiv_rn(__fmul_rn(hp.lr, m), __fsqrt_rn(__fadd_rn(vh, hp.eps))));
 }
 
-// gbar = (float)(sum over workers, accumulated in binary64) / (float)n  (Algorithm 2, line 12).
+// gbar = (float)(sum over workers, accumulated in binary64) / (float)n  (Algorithm 2, the server's average).
 // For n a power of two the division is a multiplication by the exactly representable 1 / n: both
 // round the same real number once, so the bits agree (subnormal results included) and the
 // multi-instruction IEEE division is saved.

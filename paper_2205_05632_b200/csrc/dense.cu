@@ -1,12 +1,12 @@
 // Uncompressed mode (k = d, q = 0 in Assumption 1) and the stand-alone AMSGrad update.
 //
-// dense_mean_amsgrad: gbar = mean over workers of g_i (Algorithm 2, line 12 with C = identity,
-// so e stays 0), fused with the AMSGrad update (lines 13-16). One pass over G [n, d] and the
+// dense_mean_amsgrad: gbar = mean over workers of g_i (Algorithm 2, the server's average with C = identity,
+// so e stays 0), fused with the AMSGrad update (the moment, maximum and parameter updates). One pass over G [n, d] and the
 // four state vectors: (4n + 32) bytes per coordinate plus 4 for gbar.
 //
 // amsgrad_bucket: the server update of the Top-k path. The scatter kernel has grouped the kept
 // (coordinate, value) entries of all workers by coordinate range; one CTA per range sums them in
-// binary64 in shared memory, rounds, divides by n and applies lines 13-16.
+// binary64 in shared memory, rounds, divides by n and applies the moment, maximum and parameter updates.
 #include "context.h"
 
 namespace compams {
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(kThreads, CTAS_PER_SM) dense_mean_amsgrad_kern
 
 // Server update of the Top-k path, one CTA per bucket of kBucketSpan coordinates: the bucket's kept
 // entries (all workers) are summed in binary64 in shared memory - exact, hence independent of the
-// order - then gbar = (float)sum / n and Algorithm 2, lines 13-16. Entries that did not fit their
+// order - then gbar = (float)sum / n and Algorithm 2, the moment, maximum and parameter updates. Entries that did not fit their
 // bucket were added to acc[] by the scatter kernel and are folded in (and acc cleared) here.
 __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, TopkBuffers b, float* __restrict__ theta,
                                                                      HyperParams hp) {

@@ -9,7 +9,7 @@
 //
 //   Larger blocks, cut into tiles of kTile coordinates.
 //   Candidate path (one pass over [n, d]):
-//     topk_sweep    x = g + e written over E (Algorithm 2, line 7); every key >= tau_hat, a threshold
+//     topk_sweep    x = g + e written over E (Algorithm 2, the corrected-gradient step); every key >= tau_hat, a threshold
 //                   predicted from the previous step, is appended to the segment's candidate list
 //     topk_select   if the list holds at least k_b and at most its capacity, the exact Top-k is inside it.
 //                   A histogram of the key offsets above tau_hat (bins sized from the last step) finds
@@ -27,7 +27,7 @@
 //     ties          takes the lowest-index threshold ties, tile by tile in index order
 //   topk_scatter    closes the step per segment (count check, counters reset) and walks the
 //                   (index, value) messages: each pair is appended to the bucket of its coordinate range
-//                   for the server kernel (line 12) and marked in the kept map: its e is 0 (line 8:
+//                   for the server kernel (the server's average) and marked in the kept map: its e is 0 (the residual update:
 //                   e = x - x), applied when E is next read (next sweep, or topk_materialize)
 #include <cooperative_groups.h>
 
@@ -115,7 +115,7 @@ __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float*
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
             const int r = lane_r(r0, warp, bt * NB + u, lane);
-            // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, line 8).
+            // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, the residual update).
             // Placed after the batch's loads have been issued: the shuffle waits for the map word.
             const uint32_t kb4 =
                 (__shfl_sync(0xffffffffu, mapw, (bt * NB + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
@@ -123,7 +123,7 @@ __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float*
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const float ek = ((kb4 >> k) & 1u) ? 0.0f : lane_elem(ev[u], k);
-                xs[k] = __fadd_rn(lane_elem(gv[u], k), ek);  // line 7: x = g + e
+                xs[k] = __fadd_rn(lane_elem(gv[u], k), ek);  // the corrected-gradient step: x = g + e
                 if ((FULL || (unsigned)(r + k) < (unsigned)len) && mag_key(xs[k]) >= tau_hat) {
                     const uint2 cv = make_uint2(coord0 + (uint32_t)(r + k), __float_as_uint(xs[k]));
                     const uint32_t slot = atomicAdd(sh_cnt, 1u);
@@ -1156,7 +1156,7 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
         }
     }
     if (threadIdx.x == 0 && total != kb) atomicOr(b.status, 1u);
-    // Algorithm 2, line 8: e = x - g~ (0 where kept, x elsewhere)
+    // Algorithm 2, the residual update: e = x - g~ (0 where kept, x elsewhere)
     for (int r = threadIdx.x; r < len; r += kThreads) e[r] = kept(r) ? 0.0f : __uint_as_float(xs[r]);
 }
 
@@ -1207,7 +1207,7 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
         atomicAdd(b.acc + j, (double)__uint_as_float(xbits));
         b.bdirty[T] = 1u;
     }
-    // the coordinate's e becomes 0 (line 8: e = x - x): recorded in the kept map, applied when E is next read
+    // the coordinate's e becomes 0 (the residual update: e = x - x): recorded in the kept map, applied when E is next read
     // (`count` covers the messages of every worker the server averages over; E and the kept map hold
     // the t.n workers of this handle, whose first is worker row0)
     const int64_t il = p / b.K - row0;
@@ -1216,7 +1216,7 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
     atomicOr(b.kept_cur + (size_t)(f >> 5), 1u << (uint32_t)(f & 31));
 }
 
-// E holds x at the coordinates kept in the last step: zero them (Algorithm 2, line 8), one thread per word.
+// E holds x at the coordinates kept in the last step: zero them (Algorithm 2, the residual update), one thread per word.
 __global__ void __launch_bounds__(kThreads) topk_materialize_kernel(int64_t nd, int64_t map_words,
                                                                     const uint32_t* __restrict__ kept,
                                                                     float* __restrict__ E) {

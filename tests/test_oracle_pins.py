@@ -194,7 +194,7 @@ def test_q_deviate_bound(comp):
             assert err <= q2 * np.sum(X[i, lo:hi] ** 2) * (1 + 1e-6)
 
 
-# ---------------------------------------------------------------- error feedback (Algorithm 2, lines 7-8)
+# ---------------------------------------------------------------- error feedback (Algorithm 2, the corrected-gradient and residual steps)
 
 @pytest.mark.parametrize("comp", [TOPK, BLOCKSIGN])
 def test_error_feedback_conservation_over_steps(comp):

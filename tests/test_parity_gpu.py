@@ -402,7 +402,7 @@ def test_restored_state_continues_bit_identically(comp, ratio):
     theta_saved = theta_a.clone()
     for g in G[3:]:
         a.step(g, theta_a)
-    # the saved e is what line 8 defines, not the library's deferred form of it
+    # the saved e is what the residual update defines, not the library's deferred form of it
     b = CompAMS(n, d, offs, comp, ratio)
     b.set_state(saved)
     if not (comp == TOPK and ratio == 1.0):
