@@ -116,6 +116,8 @@ __global__ void __launch_bounds__(kThreads, 8) bs_sweep_kernel(Tables t, BsBuffe
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     __shared__ uint32_t sh_first[kWarps];
+    dependency_wait();  // on small problems launched as a programmatic dependent of the step before (whose server
+                        // kernel still reads the sign words this kernel is about to overwrite)
     allow_dependents();
     const int tile = blockIdx.x;
     const int i = blockIdx.y;
@@ -306,6 +308,13 @@ static BsBuffers own_rows(const compams_context* c) {
 
 cudaError_t launch_bs_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
+    if (c->chain) {  // small problem: the launch overlaps the tail of whatever kernel precedes it on the stream
+        if (c->grad_bf16)
+            return launch_after(bs_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                                (const bf16_bits*)grads, c->e_is_x ? 1 : 0, c->segp);
+        return launch_after(bs_sweep_kernel<float>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                            (const float*)grads, c->e_is_x ? 1 : 0, c->segp);
+    }
     if (c->grad_bf16)
         bs_sweep_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads,
                                                                      c->e_is_x ? 1 : 0, c->segp);
