@@ -1,18 +1,22 @@
 #!/usr/bin/env python
 """Benchmark of the COMP-AMS optimizer step on B200.
 
-One benchmark "step" is one pass over the whole hot path on one batch of synthetic gradients
-shaped like a ResNet-18 (n = 16 workers, d = 11,173,962): one Block-Sign step (62 blocks, one
-per tensor), one whole-vector Top-k step (k = 1% of d) and one uncompressed step (k = d), each an
-optimizer of its own with its own theta and state. The metric is gradient elements consumed
-per second (n*d per optimizer step, three optimizer steps per benchmark step).
+One benchmark "step" is one optimizer step (Algorithm 2: every worker's x = g + e, compression, residual;
+the server's average and AMSGrad update) of ONE compressor on one batch of synthetic gradients. The
+headline workload is the largest single-GPU point of the scaling sweep: one block, d = 2^27 parameters,
+n = 32 workers, gradients N(0,1), Top-k with k = 1 % of d. The metric is gradient elements consumed per
+second (n d per step). Beside the headline the line carries, under "configs", one timed entry per
+workload and compressor: C1 (n=4, d=65,536), C2 / C3 (ResNet-18 shapes, n=16: Block-Sign per tensor,
+whole-vector Top-k at 0.1 % and 1 %), C4 (ResNet-50 shapes, n=32: layer-wise Top-k and Block-Sign) and the
+scaling sweep C5 (d = 2^20 .. 2^27, n = 1, 8, 32, Top-k / Block-Sign / k = d), each with its step time,
+its compulsory HBM bytes and the fraction of the HBM roofline that makes.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--only NAME ...]
 
-Prints ONE JSON line. With --gpus N > 1 (under torch.distributed.run) every rank runs an
-independent replica on its own GPU ("replicas only": the path has no inter-GPU exchange) and the
-line reports the aggregate over the max time across ranks. --impl reference times the CPU oracle
-on the host cores instead of the CUDA library.
+Prints ONE JSON line. With --gpus N > 1 (under torch.distributed.run) every rank runs an independent
+replica of the headline on its own GPU ("replicas only": the path has no inter-GPU exchange) and the line
+reports the aggregate over the max time across ranks. --impl reference times the CPU oracle on the host
+cores, on a bounded sample of the headline workload, instead of the CUDA library.
 """
 from __future__ import annotations
 
@@ -36,11 +40,19 @@ from paper_2205_05632_b200 import workloads as W
 
 METRIC = "COMP-AMS step: gradient elems/s"
 UNIT = "elem/s"
-MODES = ("blocksign", "topk", "dense")
+L2_BYTES = 126 * 1024 * 1024
+NORTH_STAR_PEAK_GBS = 8000.0  # the nominal HBM3e figure the target fraction is quoted against
+
+# kernels of each mode, the first one the dominant (the pass over [n, d])
+KERNELS = {
+    "topk": ["topk_sweep", "topk_select", "topk_dense", "topk_scatter", "amsgrad", "topk_small"],
+    "sign": ["bs_sweep", "bs_scales", "bs_apply"],
+    "dense": ["dense_mean_amsgrad"],
+}
 
 
 def measured_peak_gbs():
-    """HBM copy bandwidth measured on this machine (GB/s) and where the figure comes from."""
+    """Measured HBM copy bandwidth (GB/s) from MEASURED_PEAKS.json beside this file, else the fallback figure."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(p) as f:
@@ -49,14 +61,12 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
-# profiles/dram_traffic_bench_resnet18_n16.md, with a hash of the kernel's source code (comments and
-# white space aside) at the time of the capture: once the code changes the figure no longer describes the
-# kernel and None is reported.
-TRAFFIC = {
-    "bs_sweep": (2117579264, "blocksign.cu", "9447bdcb42baf658"),
-    "topk_sweep": (2162749952, "topk.cu", "611f9fcc91e294db"),
-    "dense_mean_amsgrad": (1144333312, "dense.cu", "c419baa10259b243"),
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per worker-element of one launch of the dominant
+# kernel, from an ncu capture of a smaller case of the same kernel (d = 2^24, n = 8; the traffic of these
+# streaming kernels grows in proportion to n d), with a hash of the kernel's source code (comments and white
+# space aside) at the time of the capture: once the code changes the figure no longer describes the kernel and
+# None is reported.
+TRAFFIC_PER_ELEM = {
 }
 
 
@@ -74,35 +84,29 @@ def code_hash(paths):
     return hashlib.sha256(text.encode()).hexdigest()[:16]
 
 
-def captured_traffic(kernel: str):
-    if kernel not in TRAFFIC:
+def captured_traffic(kernel: str, elems: int):
+    if kernel not in TRAFFIC_PER_ELEM:
         return None
-    nbytes, src, want = TRAFFIC[kernel]
+    per_elem, src, want = TRAFFIC_PER_ELEM[kernel]
     base = os.path.join(ROOT, "paper_2205_05632_b200", "csrc")
     try:
         have = code_hash([os.path.join(base, src), os.path.join(base, "common.cuh")])
     except OSError:
         return None
-    return nbytes if have == want else None
+    return int(per_elem * elems) if have == want else None
 
 
-def min_bytes(mode: str, n: int, d: int) -> int:
-    """Compulsory HBM bytes of one optimizer step: g and e read, e written (12 B per worker-element),
-    m, v, vhat, theta read and written (32 B per coordinate); k = d never touches e."""
-    return (4 * n + 32) * d if mode == "dense" else (12 * n + 32) * d
+def min_bytes(mode: str, n: int, d: int, bf16: bool = False) -> int:
+    """Compulsory HBM bytes of one optimizer step: g and e read, e written (12 B per worker-element, 10 B
+    with bfloat16 gradients), m, v, vhat, theta read and written (32 B per coordinate); k = d never touches e."""
+    g = 2 if bf16 else 4
+    return (g * n + 32) * d if mode == "dense" else ((g + 8) * n + 32) * d
 
 
-def build_workloads(device):
-    """The three optimizers' inputs: two pre-generated gradient batches each (a ring), theta_1."""
-    out = {}
-    specs = {"blocksign": W.config2(device), "topk": W.config3(0.01, device)}
-    for mode, w in specs.items():
-        theta = w.start()
-        out[mode] = dict(w=w, theta=theta, grads=[w.grads(), w.grads()])
-    # the uncompressed step consumes the Block-Sign optimizer's gradients (same shapes, k = d)
-    wd = W.config3(1.0, device)
-    out["dense"] = dict(w=wd, theta=out["blocksign"]["theta"].clone(), grads=out["blocksign"]["grads"])
-    return out
+def algorithmic_bytes(kernel: str, n: int, d: int) -> int:
+    """Bytes one launch of a dominant kernel must move: the sweeps read g and e and write x (12 B per
+    worker-element, plus one sign bit for Block-Sign); the k = d kernel reads g and updates the state."""
+    return {"bs_sweep": 12 * n * d + n * d // 8, "topk_sweep": 12 * n * d, "dense_mean_amsgrad": (4 * n + 36) * d}[kernel]
 
 
 class ClockSampler:
@@ -156,82 +160,186 @@ class ClockSampler:
         return out
 
 
-def time_oracle(wl, steps: int, warmup: int, workers=None):
-    """Times the CPU oracle, as it stands, on the same workload (optionally only the first `workers`
-    worker rows of it): seconds per benchmark step and the threads it used."""
+# ------------------------------------------------------------------------------------------------------
+# workloads
+
+def headline_point(device) -> dict:
+    """The largest single-GPU point of the scaling sweep that fits the device: d = 2^27, n = 32 needs about
+    75 GB (two gradient batches, E, the end-to-end staging buffer); smaller devices take d = 2^26."""
+    lg = 27
+    if device != "cpu":
+        free, _ = torch.cuda.mem_get_info()
+        if free < 85 * (1 << 30):
+            lg = 26
+    return dict(config="C5", mode="topk", n=32, log2d=lg)
+
+
+def describe(pt) -> str:
+    return ("scaling sweep (C5) largest single-GPU point: one block, d = 2^%d, n = %d workers, gradients i.i.d. "
+            "N(0,1), Top-k with k = 1%% of d; one optimizer step per benchmark step" % (pt["log2d"], pt["n"]))
+
+
+def workload_config(pt):
+    n, d = pt["n"], 1 << pt["log2d"]
+    return {
+        "workload": describe(pt), "n_workers": n, "d": d, "compressor": "topk", "k_ratio": 0.01,
+        "l2": "inputs larger than L2 (each [n,d] buffer is %.1f GB; ring of 2 gradient batches)" % (n * d * 4 / 1e9),
+        "parallelism": "replicas only",
+    }
+
+
+def config_entries():
+    """Every timed entry of "configs": (name, builder of the workload on a device, mode, bfloat16 input)."""
+    out = [("C1/topk1%", lambda dev: W.config1(dev), "topk", False),
+           ("C2/sign", lambda dev: W.config2(dev), "sign", False),
+           ("C2/sign/bf16", lambda dev: W.config2(dev), "sign", True),
+           ("C3/topk0.1%", lambda dev: W.config3(0.001, dev), "topk", False),
+           ("C3/topk1%", lambda dev: W.config3(0.01, dev), "topk", False),
+           ("C3/topk1%/bf16", lambda dev: W.config3(0.01, dev), "topk", True),
+           ("C4/topk1%/layerwise", lambda dev: W.config4(W.TOPK, dev), "topk", False),
+           ("C4/sign", lambda dev: W.config4(W.BLOCKSIGN, dev), "sign", False)]
+    for lg in (20, 22, 24, 26, 27):
+        for n in (1, 8, 32):
+            for mode in ("topk", "sign", "dense"):
+                out.append(("C5/%s/d=2^%d/n=%d" % (mode, lg, n),
+                            (lambda dev, lg=lg, n=n, mode=mode: W.sweep_point(1 << lg, n, mode, dev)), mode, False))
+    return out
+
+
+def time_entry(name, build, mode, bf16, steps, warmup, peak, peak_kind, cache):
+    """Creates the workload and its optimizer, runs `warmup` + `steps` steps and returns the entry's record."""
+    from paper_2205_05632_b200 import CompAMS
+    w = build("cuda")
+    key = (w.n, w.d, name.split("/")[0], bf16)
+    if key in cache:  # the modes of one sweep point consume the same gradients
+        theta0, ring = cache[key]
+    else:
+        cache.clear()
+        torch.cuda.empty_cache()
+        theta0 = w.start()
+        ring = [w.grads(), w.grads()]
+        if bf16:
+            ring = [g.bfloat16() for g in ring]
+        cache[key] = (theta0, ring)
+    theta = theta0.clone()
+    opt = CompAMS(w.n, w.d, w.block_offsets, w.compressor, w.k_ratio, w.lr, w.beta1, w.beta2, w.eps)
+    try:
+        for t in range(warmup):
+            opt.step(ring[t % 2], theta)
+        opt.check_status()
+        st0 = opt.buffer("status").cpu().tolist()
+        l0 = opt.launch_count()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        s.record()
+        for t in range(steps):
+            opt.step(ring[(warmup + t) % 2], theta)
+        e.record()
+        torch.cuda.synchronize()
+        opt.check_status()
+        ms = s.elapsed_time(e) / steps
+        st1 = opt.buffer("status").cpu().tolist()
+        launches = (opt.launch_count() - l0) / steps
+    finally:
+        opt.close()
+    mb = min_bytes(mode, w.n, w.d, bf16)
+    gbs = mb / ms / 1e6
+    fits_l2 = 2 * w.n * w.d * 4 <= L2_BYTES
+    rec = {"name": name, "mode": mode, "n": w.n, "d": w.d, "blocks": int(len(w.block_offsets) - 1),
+           "ms": ms, "elems_per_s": w.n * w.d / ms * 1e3, "min_bytes": mb, "launches_per_step": launches}
+    if fits_l2:
+        rec["note"] = "launch-bound: inputs fit L2, no HBM fraction"
+    else:
+        rec.update({"hbm_gbs": gbs, "frac_of_%s" % peak_kind: gbs / peak, "frac_of_8TBs": gbs / NORTH_STAR_PEAK_GBS})
+    if mode == "topk":
+        # selections of the timed steps decided by the dense passes / inside the candidate lists, and why lists
+        # were given up (too few, too many, out of range, crowded threshold bin)
+        rec["status"] = {"word": st1[0], "dense": st1[1] - st0[1], "candidate": st1[2] - st0[2],
+                         "gave_up": [st1[k] - st0[k] for k in (3, 4, 5, 6)]}
+    return rec
+
+
+# ------------------------------------------------------------------------------------------------------
+# the oracle on the host cores
+
+def oracle_sample(pt, rows_gpu=None, budget_s=20.0, steps=None, warmup=1):
+    """Times the CPU oracle, as it stands, on a bounded sample of the headline workload: the first `ns`
+    worker rows over the first `ds` coordinates (one block), shrunk until the run fits its time budget.
+    Returns (elements per second, threads, description, seconds per step, steps timed)."""
     import oracle
     cores = oracle.max_threads()
-    refs = {}
-    for mode in MODES:
-        w = wl[mode]["w"]
-        ns = w.n if workers is None else min(workers, w.n)
-        refs[mode] = dict(o=oracle.Oracle(ns, w.d, w.block_offsets, w.compressor, w.k_ratio, w.lr, w.beta1, w.beta2,
-                                          w.eps),
-                          theta=wl[mode]["theta"].cpu().numpy().copy(),
-                          grads=[np.ascontiguousarray(g[:ns].cpu().numpy()) for g in wl[mode]["grads"]])
+    n, d = pt["n"], 1 << pt["log2d"]
+    ns, ds = min(n, max(1, cores), 8), d
 
-    def one(t):
-        for mode in MODES:
-            r = refs[mode]
-            r["o"].step(r["grads"][t % 2], r["theta"])
+    def rows(ns_, ds_):
+        if rows_gpu is not None:
+            return np.ascontiguousarray(rows_gpu[:ns_, :ds_].cpu().numpy())
+        gen = torch.Generator().manual_seed(0)
+        return torch.randn(ns_, ds_, generator=gen, dtype=torch.float32).numpy()
 
-    for t in range(warmup):
-        one(t)
+    while True:
+        G = rows(ns, ds)
+        o = oracle.Oracle(ns, ds, [0, ds], oracle.TOPK, 0.01)
+        theta = np.zeros(ds, dtype=np.float32)
+        t0 = time.perf_counter()
+        o.step(G, theta)
+        probe = time.perf_counter() - t0
+        want_steps = steps if steps is not None else max(2, int(budget_s / max(probe, 1e-6)))
+        total = probe * (want_steps + warmup)
+        if steps is None or total <= budget_s or (ns == 1 and ds <= (1 << 20)):
+            break
+        o.close()
+        # too slow for the budget: fewer rows first (they run in parallel up to the core count), then fewer coordinates
+        if ns > 1:
+            ns = 1
+        else:
+            ds = max(1 << 20, ds // 4)
+    if steps is None:
+        want_steps = min(want_steps, 20)
+    for _ in range(max(0, warmup - 1)):
+        o.step(G, theta)
     t0 = time.perf_counter()
-    for t in range(steps):
-        one(warmup + t)
-    dt = (time.perf_counter() - t0) / max(steps, 1)
-    for r in refs.values():
-        r["o"].close()
-    return dt, cores
+    for _ in range(want_steps):
+        o.step(G, theta)
+    dt = (time.perf_counter() - t0) / want_steps
+    o.close()
+    what = ("the first %d of %d worker rows%s of the headline workload, Top-k 1%%; %d steps after %d warm-up" % (
+        ns, n, "" if ds == d else " over the first %d of %d coordinates" % (ds, d), want_steps, warmup))
+    return ns * ds / dt, cores, what, dt, want_steps
 
 
 def run_reference(args):
     """--impl reference: the oracle on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    wl = build_workloads("cpu")
-    n, d = wl["topk"]["w"].n, wl["topk"]["w"].d
-    # bounded sample: as many of the n worker rows as keep the whole run near two minutes
-    probe, _ = time_oracle(wl, 1, 1, workers=1)
-    per_step = 120.0 / max(args.steps + args.warmup, 1)
-    ns = int(max(1, min(n, per_step / max(probe, 1e-9))))
-    dt, cores = time_oracle(wl, args.steps, args.warmup, workers=ns)
-    elems = len(MODES) * ns * d
-    value = elems / dt
+    pt = dict(config="C5", mode="topk", n=32, log2d=27)
+    value, cores, what, dt, _ = oracle_sample(pt, None, budget_s=150.0, steps=args.steps, warmup=max(args.warmup, 1))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_config(n, d),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": "the first %d of %d worker rows of the workload, every coordinate; %d steps "
-                                   "after %d warm-up" % (ns, n, args.steps, args.warmup)},
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(pt),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
 
 
-def workload_config(n, d):
-    return {
-        "workload": "ResNet-18-shaped gradients (62 tensors, d=%d), n=%d workers: per step one Block-Sign step "
-                    "(one block per tensor; Student-t(3) x fan_in^-1/2), one whole-vector Top-k step (k=1%% of d; "
-                    "same values with 5%% exact zeros) and one uncompressed step (k=d)" % (d, n),
-        "n_workers": n, "d": d, "optimizer_steps_per_step": len(MODES),
-        "l2": "inputs larger than L2 (each [n,d] buffer is %.0f MB; ring of 2 gradient batches)" % (n * d * 4 / 1e6),
-        "parallelism": "replicas only",
-    }
-
+# ------------------------------------------------------------------------------------------------------
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (rank 0, N=1)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration entries")
+    ap.add_argument("--no-headline", action="store_true", help="time only the entries selected with --only")
+    ap.add_argument("--only", nargs="*", default=None, help="names (or prefixes) of the 'configs' entries to time")
+    ap.add_argument("--config-steps", type=int, default=20)
+    ap.add_argument("--config-warmup", type=int, default=8)
+    ap.add_argument("--e2e-steps", type=int, default=3)
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -240,136 +348,129 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the COMP-AMS library has no CPU path")
-    from paper_2205_05632_b200 import CompAMS
+    from paper_2205_05632_b200 import CompAMS, replicas
 
-    from paper_2205_05632_b200 import replicas
     rank, world, local = replicas.rank_world_local()
     torch.cuda.set_device(local)
     dist = replicas.init("nccl", torch.device("cuda", local))
-
     device = "cuda"
-    wl = build_workloads(device)
-    n, d = wl["topk"]["w"].n, wl["topk"]["w"].d
-    stream = torch.cuda.current_stream()
-    opts = {}
-    for mode in MODES:
-        w = wl[mode]["w"]
-        opts[mode] = CompAMS(w.n, w.d, w.block_offsets, w.compressor, w.k_ratio, w.lr, w.beta1, w.beta2, w.eps,
-                             stream=stream)
-    dominant = {"blocksign": "bs_sweep", "topk": "topk_sweep", "dense": "dense_mean_amsgrad"}
-
-    def one_step(t):
-        for mode in MODES:
-            opts[mode].step(wl[mode]["grads"][t % 2], wl[mode]["theta"])
-
-    def barrier():
-        replicas.barrier(dist)
-
-    for t in range(args.warmup):
-        one_step(t)
-    for mode in MODES:
-        opts[mode].check_status()
-        opts[mode].set_profiling([dominant[mode]])
-    launches0 = sum(o.launch_count() for o in opts.values())
-
-    # ---- timed region: K steps, device time from CUDA events on the launching stream
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(MODES) + 1)]
-    mode_ms = {m: 0.0 for m in MODES}
-    barrier()
-    sampler = ClockSampler(local)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    per_step_events = []
-    start.record(stream)
-    for t in range(args.steps):
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(MODES) + 1)]
-        evs[0].record(stream)
-        for k, mode in enumerate(MODES):
-            opts[mode].step(wl[mode]["grads"][(args.warmup + t) % 2], wl[mode]["theta"])
-            evs[k + 1].record(stream)
-        per_step_events.append(evs)
-    stop.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    elapsed_ms = start.elapsed_time(stop)
-    for evs in per_step_events:
-        for k, mode in enumerate(MODES):
-            mode_ms[mode] += evs[k].elapsed_time(evs[k + 1])
-    launches = sum(o.launch_count() for o in opts.values()) - launches0
-    for o in opts.values():
-        o.check_status()
-
-    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, device)
-    ms_per_step = elapsed_ms / args.steps
-    elems_per_step = len(MODES) * n * d
-    value = replicas.aggregate_throughput(elems_per_step, world, ms_per_step)
-
-    # ---- roofline of the dominant kernel, live from the event pairs recorded in the timed region
     peak, peak_kind = measured_peak_gbs()
-    kern = {}
-    for mode in MODES:
-        ms, cnt = opts[mode].kernel_time(dominant[mode])
-        kern[dominant[mode]] = (ms, cnt)
-    top = max(kern, key=lambda k: kern[k][0])
-    # algorithmic bytes per launch of the sweeps: g and e read, x/e written = 12 B per worker-element
-    # (+ n*d/8 sign-bit bytes for Block-Sign); dense: (4n + 36) B per coordinate
-    alg = {"bs_sweep": 12 * n * d + n * d // 8, "topk_sweep": 12 * n * d, "dense_mean_amsgrad": (4 * n + 36) * d}
-    top_ms = kern[top][0] / max(kern[top][1], 1)
-    achieved = alg[top] / (top_ms * 1e-3) / 1e9
-    roofline = {"kernel": top, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": captured_traffic(top),
-                "avg_launch_ms": top_ms, "launches_timed": kern[top][1],
-                "algorithmic_bytes_per_launch": alg[top]}
-    per_kernel = {k: {"avg_ms": v[0] / max(v[1], 1), "launches": v[1],
-                      "achieved_gbs": alg[k] / (v[0] / max(v[1], 1) * 1e-3) / 1e9 if v[0] > 0 else None}
-                  for k, v in kern.items()}
+    stream = torch.cuda.current_stream()
+    line = {}
 
-    # ---- whole optimizer steps against their compulsory traffic
-    modes_out = {}
-    for mode in MODES:
-        ms = mode_ms[mode] / args.steps
-        bmin = min_bytes(mode, n, d)
-        gbs = bmin / (ms * 1e-3) / 1e9
-        modes_out[mode] = {"ms": ms, "elems_per_s": n * d / (ms * 1e-3), "steps_per_s": 1e3 / ms,
-                           "min_bytes": bmin, "hbm_gbs": gbs, "frac_of_%s_peak" % peak_kind: gbs / peak,
-                           "frac_of_8TBs": gbs / 8000.0}
+    if not args.no_headline:
+        pt = headline_point(device)
+        n, d = pt["n"], 1 << pt["log2d"]
+        w = W.sweep_point(d, n, "topk", device)
+        theta = w.start()
+        ring = [w.grads(), w.grads()]
+        opt = CompAMS(w.n, w.d, w.block_offsets, w.compressor, w.k_ratio, w.lr, w.beta1, w.beta2, w.eps, stream=stream)
+        # at least three warm-up steps: the first selections run the dense passes, the threshold prediction
+        # carries the rest
+        for t in range(max(args.warmup, 3)):
+            opt.step(ring[t % 2], theta)
+        opt.check_status()
+        st0 = opt.buffer("status").cpu().tolist()
+        opt.set_profiling(["topk_sweep"])
+        launches0 = opt.launch_count()
 
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": workload_config(n, d),
-        "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "kernels": per_kernel, "modes": modes_out,
-    }
+        # ---- timed region: K steps, device time from CUDA events on the launching stream
+        replicas.barrier(dist)
+        sampler = ClockSampler(local)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(stream)
+        for t in range(args.steps):
+            opt.step(ring[(args.warmup + t) % 2], theta)
+        stop.record(stream)
+        replicas.barrier(dist)
+        clocks = sampler.stop()
+        elapsed_ms = start.elapsed_time(stop)
+        launches = opt.launch_count() - launches0
+        opt.check_status()
+        st1 = opt.buffer("status").cpu().tolist()
+        sweep_ms, sweep_cnt = opt.kernel_time("topk_sweep")
 
-    # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
-    if not args.no_e2e:
-        for o in opts.values():
-            o.set_profiling([])
-        host = {m: dict(g=[g.cpu().pin_memory() for g in wl[m]["grads"]], th=wl[m]["theta"].cpu().pin_memory())
-                for m in ("blocksign", "topk")}
-        host["dense"] = dict(g=host["blocksign"]["g"], th=wl["dense"]["theta"].cpu().pin_memory())
-        for mode in MODES:  # allocate the staging buffers outside the timed region
-            opts[mode].step_host(host[mode]["g"][0], host[mode]["th"])
-        barrier()
-        t0 = time.perf_counter()
-        for t in range(args.e2e_steps):
-            for mode in MODES:
-                opts[mode].step_host(host[mode]["g"][t % 2], host[mode]["th"])
-        torch.cuda.synchronize()
-        dt = (time.perf_counter() - t0) / args.e2e_steps
-        dt = replicas.max_over_ranks(dt, dist, device)
-        line["e2e"] = {"value": world * elems_per_step / dt, "unit": UNIT, "ms_per_step": dt * 1e3,
-                       "h2d_bytes_per_step": len(MODES) * (n * d * 4 + d * 4),
-                       "d2h_bytes_per_step": len(MODES) * d * 4, "steps": args.e2e_steps,
-                       "call": "compams_step_host (pinned host buffers, synchronous)"}
+        elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, device)
+        ms_per_step = elapsed_ms / args.steps
+        value = replicas.aggregate_throughput(n * d, world, ms_per_step)
 
-    # ---- the oracle on the host cores, rank 0 at N = 1 only
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dt, cores = time_oracle(wl, 20, 1)
-        line["cpu_baseline"] = {"value": elems_per_step / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "ms_per_step": dt * 1e3,
-                                "sample": "20 steps of the full workload (all %d workers) after 1 warm-up step" % n}
-    for o in opts.values():
-        o.close()
+        # ---- roofline: the dominant kernel live from the event pairs of the timed region, and the whole step
+        # against its compulsory bytes
+        alg = algorithmic_bytes("topk_sweep", n, d) * args.steps  # every step sweeps all n rows (in one or more launches)
+        achieved = alg / (sweep_ms * 1e-3) / 1e9 if sweep_ms > 0 else None
+        mb = min_bytes("topk", n, d)
+        step_gbs = mb / (ms_per_step * 1e-3) / 1e9
+        roofline = {"kernel": "topk_sweep", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak if achieved else None, "peak_kind": "of " + peak_kind,
+                    "traffic": captured_traffic("topk_sweep", n * d),
+                    "avg_launch_ms": sweep_ms / max(sweep_cnt, 1), "launches_timed": sweep_cnt,
+                    "algorithmic_bytes_per_step": alg // args.steps,
+                    "step_min_bytes": mb, "step_gbs": step_gbs, "step_frac": step_gbs / peak,
+                    "step_frac_of_8TBs": step_gbs / NORTH_STAR_PEAK_GBS}
+
+        # ---- per-kernel breakdown of the step, from a few extra steps with an event pair around every launch
+        opt.set_profiling(KERNELS["topk"])
+        for t in range(3):
+            opt.step(ring[t % 2], theta)
+        per_kernel = {}
+        for k in KERNELS["topk"]:
+            ms, cnt = opt.kernel_time(k)
+            if cnt:
+                per_kernel[k] = {"ms_per_step": ms / 3, "launches_per_step": cnt / 3}
+        opt.set_profiling([])
+
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "steps_per_s": 1e3 / ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(pt),
+            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "kernels": per_kernel,
+            "status": {"word": st1[0], "dense": st1[1] - st0[1], "candidate": st1[2] - st0[2],
+                       "gave_up": [st1[k] - st0[k] for k in (3, 4, 5, 6)]},
+        }
+
+        # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
+        if not args.no_e2e:
+            del ring[1]
+            torch.cuda.empty_cache()
+            hg = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+            hg.copy_(ring[0])
+            ht = torch.empty(d, dtype=torch.float32, pin_memory=True)
+            ht.copy_(theta)
+            opt.step_host(hg, ht)  # allocates the staging buffers outside the timed region
+            replicas.barrier(dist)
+            t0 = time.perf_counter()
+            for t in range(args.e2e_steps):
+                opt.step_host(hg, ht)
+            torch.cuda.synchronize()
+            dt = (time.perf_counter() - t0) / args.e2e_steps
+            dt = replicas.max_over_ranks(dt, dist, device)
+            line["e2e"] = {"value": world * n * d / dt, "unit": UNIT, "ms_per_step": dt * 1e3,
+                           "h2d_bytes_per_step": n * d * 4 + d * 4, "d2h_bytes_per_step": d * 4,
+                           "steps": args.e2e_steps, "call": "compams_step_host (pinned host buffers, synchronous)"}
+            del hg, ht
+
+        # ---- the oracle on the host cores, rank 0 at N = 1 only
+        if rank == 0 and world == 1 and not args.no_cpu_baseline:
+            v, cores, what, dt, _ = oracle_sample(pt, ring[0], budget_s=20.0)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "ms_per_step": dt * 1e3,
+                                    "sample": what}
+        opt.close()
+        del ring, theta
+        torch.cuda.empty_cache()
+
+    # ---- every configuration, one compressor per number (rank 0 at N = 1 only)
+    if rank == 0 and world == 1 and not args.no_configs:
+        entries, cache = [], {}
+        for name, build, mode, bf16 in config_entries():
+            if args.only is not None and not any(name.startswith(p) for p in args.only):
+                continue
+            entries.append(time_entry(name, build, mode, bf16, args.config_steps, args.config_warmup, peak, peak_kind,
+                                      cache))
+        cache.clear()
+        line["configs"] = entries
+        line["configs_protocol"] = ("per entry: %d steps between two CUDA events after %d warm-up steps, ring of 2 gradient "
+                                    "batches; min_bytes = (12 n + 32) d with error feedback ((10 n + 32) d with bfloat16 "
+                                    "gradients), (4 n + 32) d for k = d" % (args.config_steps, args.config_warmup))
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

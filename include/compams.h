@@ -18,7 +18,9 @@
  *     caller memory. All device work is enqueued on the handle's CUDA stream (default: the legacy
  *     default stream); calls return without synchronising unless stated otherwise.
  *   - Every call returns COMPAMS_OK (0) or a negative compams_status. Nothing aborts, throws or
- *     prints. One handle may be used by one host thread at a time.
+ *     prints. One handle may be used by one host thread at a time, and every call that enqueues work
+ *     on a handle must be made with the CUDA device current on which the handle was created
+ *     (otherwise: INVALID_ARG, nothing is enqueued).
  *   - All state is fp32. Every fp32 operation of the update is a separately rounded IEEE
  *     operation (no fused multiply-add, IEEE sqrt and division, subnormals kept).
  *   - Gradients must be finite. NaN/Inf make the Top-k selection undefined (no fault, but the
@@ -82,7 +84,7 @@ enum compams_kernel {
     COMPAMS_K_TOPK_DENSE = 5,         /* Top-k dense passes (one cooperative launch): radix histograms over x,
                                          threshold search, emission, lowest-index ties                        */
     COMPAMS_K_TOPK_MATERIALIZE = 6,   /* Top-k: zero e at the coordinates kept in the last step when E is read   */
-    /* 7, 8: unused */
+    /* 7, 8: reserved (never returned, never timed) */
     COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: closes the step per segment; sparse scatter-accumulate         */
     COMPAMS_K_AMSGRAD = 10,           /* Top-k: AMSGrad update from the accumulated average                   */
     COMPAMS_K_TOPK_SMALL = 11,        /* Top-k: whole small blocks selected inside shared memory              */
@@ -97,7 +99,7 @@ enum compams_kernel {
  *
  *   out            host; receives the handle. Untouched on failure.
  *   n              number of simulated workers, 1 <= n <= 65535.
- *   d              number of parameters, 1 <= d < 2^31.
+ *   d              number of parameters, 1 <= d <= 2^31 - 32768.
  *   block_offsets  host; num_blocks + 1 entries, [0] = 0, strictly increasing, last = d. Copied.
  *   num_blocks     M >= 1. The compressor acts on each block separately (Section 3.1). With one
  *                  block Top-k is taken over the whole vector; with one block per tensor it is
@@ -192,6 +194,12 @@ int compams_step_host(compams_handle h, const float* grads_host, float* theta_ho
  * compams_step on a handle with n_local == n_total is compams_compress followed by compams_apply;
  * on a sharded handle it returns INVALID_ARG (the exchange is missing). Both calls enqueue on the
  * handle's stream and return without synchronising.
+ *
+ * Order of calls: compams_compress opens an iteration and compams_apply closes it. In between the
+ * residual update of the workers is not yet final, so compams_compress, compams_step, compams_step_host,
+ * compams_get_state, compams_set_state and compams_get_buffer(BUF_E) return INVALID_ARG (the message
+ * buffers and the server's buffers stay readable); compams_apply without an open iteration returns
+ * INVALID_ARG too.
  */
 int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total, int32_t first_worker, int64_t d,
                            const int64_t* block_offsets, int32_t num_blocks, int32_t compressor, double k_ratio, float lr,

@@ -30,6 +30,8 @@ def lib() -> ctypes.CDLL:
                                     c.c_float, c.c_float, c.c_float, c.c_float]
         L.oracle_destroy.restype = None
         L.oracle_destroy.argtypes = [c.c_void_p]
+        L.oracle_set_lr.restype = None
+        L.oracle_set_lr.argtypes = [c.c_void_p, c.c_float]
         L.oracle_step.restype = c.c_int
         L.oracle_step.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
         L.oracle_buffer.restype = c.c_void_p
@@ -114,6 +116,10 @@ class Oracle:
         rc = lib().oracle_step(self._h, G.ctypes.data, theta.ctypes.data)
         if rc != 0:
             raise RuntimeError("oracle_step failed")
+
+    def set_lr(self, lr: float) -> None:
+        """eta_t of the following steps (Algorithm 2 lets the learning rate vary with t)."""
+        lib().oracle_set_lr(self._h, float(lr))
 
     def buffer(self, name: str) -> np.ndarray:
         """A view (not a copy) of an oracle buffer, valid until the next step or close()."""

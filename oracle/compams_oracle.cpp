@@ -183,6 +183,12 @@ void* oracle_create(int32_t n, int64_t d, const int64_t* block_offsets, int32_t 
 
 void oracle_destroy(void* h) { delete (Oracle*)h; }
 
+// Algorithm 2 takes a learning rate eta_t per iteration: the value set here is the eta_t of every
+// following oracle_step until it is set again (Section 5.1 divides it by 10 at fixed epochs).
+void oracle_set_lr(void* h, float lr) {
+    if (h) ((Oracle*)h)->lr = lr;
+}
+
 // One iteration t of Algorithm 2 given the workers' stochastic gradients G [n, d] (row i = g_{t,i})
 // and the server parameters theta [d], which are updated in place.
 int oracle_step(void* h, const float* G, float* theta) {

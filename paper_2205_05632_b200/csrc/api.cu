@@ -57,6 +57,14 @@ int dev_upload(compams_context* c, T** out, const std::vector<T>& host) {
         if (_rc) return _rc;  \
     } while (0)
 
+// Every enqueueing call must run with the handle's device current: its buffers live there, and on the
+// default stream a launch goes to whatever device is current.
+int on_handle_device(const compams_context* c) {
+    int dev = -1;
+    CU(cudaGetDevice(&dev));
+    return dev == c->device ? COMPAMS_OK : COMPAMS_ERR_INVALID_ARG;
+}
+
 int64_t kept_per_block(double k_ratio, int64_t d_b) {
     int64_t k = (int64_t)std::floor(k_ratio * (double)d_b);
     if (k < 1) k = 1;
@@ -133,9 +141,10 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
     c->seg_cap_host.clear();
     for (const SegInfo& si : segs) c->seg_cap_host.push_back(si.cap);
     if (topk) {
-        // Short candidate lists get one CTA each, long ones a cluster of CTAs. A cluster finishes one
-        // list sooner, but far fewer clusters than CTAs fit on the GPU at once: with many long lists
-        // (layer-wise selection over many workers) one CTA per list has the higher throughput.
+        // Short candidate lists get one CTA each; a long one is cut into slices that many CTAs work on
+        // (two kernels that meet through a global histogram). Slices finish one list sooner, but with
+        // many long lists (layer-wise selection over many workers) one CTA per list has the higher
+        // throughput.
         size_t n_long = 0;
         for (const SegInfo& si : segs) n_long += si.cap > (uint32_t)kSelectSingleMax ? 1 : 0;
         const uint32_t single_max = (n_long * (size_t)c->n >= 64) ? (1u << 20) : (uint32_t)kSelectSingleMax;
@@ -315,9 +324,8 @@ int run_kernel(compams_context* c, int kernel, F&& launch) {
         c->ev_kernel[(size_t)slot] = kernel;
         CU(cudaEventRecord(c->ev_start[(size_t)slot], c->stream));
     }
-    cudaError_t e = launch();
+    cudaError_t e = launch();  // the launchers count the kernels they enqueue in c->launches
     if (e != cudaSuccess) return cuda_fail(e, compams_kernel_name(kernel));
-    ++c->launches;
     if (slot >= 0) CU(cudaEventRecord(c->ev_stop[(size_t)slot], c->stream));
     return COMPAMS_OK;
 }
@@ -371,7 +379,8 @@ int step_device(compams_context* c, const void* grads, float* theta) {
 int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0, int64_t d, const int64_t* block_offsets,
                   int32_t num_blocks, int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps) {
     if (!out || !block_offsets) return COMPAMS_ERR_INVALID_ARG;
-    if (n < 1 || n_total > 65535 || row0 < 0 || (int64_t)row0 + n > n_total || d < 1 || d >= ((int64_t)1 << 31) ||
+    // the tiled kernels address a block with 32-bit coordinates that may run up to two tiles past its end
+    if (n < 1 || n_total > 65535 || row0 < 0 || (int64_t)row0 + n > n_total || d < 1 || d > kMaxD ||
         num_blocks < 1 || (int64_t)num_blocks > d)
         return COMPAMS_ERR_INVALID_ARG;
     if (compressor != COMPAMS_TOPK && compressor != COMPAMS_BLOCKSIGN) return COMPAMS_ERR_INVALID_ARG;
@@ -434,12 +443,17 @@ int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total
 static int compress_any(compams_handle c, const void* grads, bool bf16) {
     if (!c || !grads || (reinterpret_cast<uintptr_t>(grads) & (bf16 ? 1u : 3u))) return COMPAMS_ERR_INVALID_ARG;
     if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;  // k = d: nothing is compressed
+    if (c->compressed) return COMPAMS_ERR_INVALID_ARG;  // the previous compress has not been applied yet
+    RC(on_handle_device(c));
     c->grad_bf16 = bf16;
+    int rc;
     try {
-        return compress_device(c, grads);
+        rc = compress_device(c, grads);
     } catch (const std::bad_alloc&) {
-        return COMPAMS_ERR_ALLOC;
+        rc = COMPAMS_ERR_ALLOC;
     }
+    if (!rc) c->compressed = true;
+    return rc;
 }
 
 int compams_compress(compams_handle c, const float* grads) { return compress_any(c, grads, false); }
@@ -448,6 +462,9 @@ int compams_compress_bf16(compams_handle c, const void* grads_bf16) { return com
 int compams_apply(compams_handle c, float* theta) {
     if (!c || !theta || (reinterpret_cast<uintptr_t>(theta) & 15u)) return COMPAMS_ERR_INVALID_ARG;
     if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;
+    if (!c->compressed) return COMPAMS_ERR_INVALID_ARG;  // nothing to apply: compams_compress comes first
+    RC(on_handle_device(c));
+    c->compressed = false;
     try {
         return apply_device(c, theta);
     } catch (const std::bad_alloc&) {
@@ -460,6 +477,8 @@ static int step_any(compams_handle c, const void* grads, float* theta, bool bf16
     if ((reinterpret_cast<uintptr_t>(grads) & (bf16 ? 1u : 3u)) || (reinterpret_cast<uintptr_t>(theta) & 15u))
         return COMPAMS_ERR_INVALID_ARG;
     if (c->n != c->n_total) return COMPAMS_ERR_INVALID_ARG;  // the other workers' messages have to be exchanged first
+    if (c->compressed) return COMPAMS_ERR_INVALID_ARG;       // a compams_compress is waiting for its compams_apply
+    RC(on_handle_device(c));
     c->grad_bf16 = bf16;
     try {
         return step_device(c, grads, theta);
@@ -472,7 +491,8 @@ int compams_step(compams_handle c, const float* grads, float* theta) { return st
 int compams_step_bf16(compams_handle c, const void* grads_bf16, float* theta) { return step_any(c, grads_bf16, theta, true); }
 
 int compams_step_host(compams_handle c, const float* grads_host, float* theta_host) {
-    if (!c || !grads_host || !theta_host || c->n != c->n_total) return COMPAMS_ERR_INVALID_ARG;
+    if (!c || !grads_host || !theta_host || c->n != c->n_total || c->compressed) return COMPAMS_ERR_INVALID_ARG;
+    RC(on_handle_device(c));
     const size_t gbytes = (size_t)c->n * (size_t)c->d * sizeof(float);
     const size_t tbytes = (size_t)c->d * sizeof(float);
     if (!c->stage_grads) {
@@ -537,8 +557,8 @@ static int finish_residual(compams_context* c) {
 }
 
 int compams_get_state(compams_handle c, float* e, float* m, float* v, float* vhat) {
-    if (!c) return COMPAMS_ERR_INVALID_ARG;
-    CU(cudaSetDevice(c->device));
+    if (!c || c->compressed) return COMPAMS_ERR_INVALID_ARG;  // between compress and apply the step is half done
+    RC(on_handle_device(c));
     const size_t nd = (size_t)c->n * (size_t)c->d * sizeof(float), db = (size_t)c->d * sizeof(float);
     if (e) {
         if (c->E) {
@@ -555,8 +575,8 @@ int compams_get_state(compams_handle c, float* e, float* m, float* v, float* vha
 }
 
 int compams_set_state(compams_handle c, const float* e, const float* m, const float* v, const float* vhat) {
-    if (!c) return COMPAMS_ERR_INVALID_ARG;
-    CU(cudaSetDevice(c->device));
+    if (!c || c->compressed) return COMPAMS_ERR_INVALID_ARG;
+    RC(on_handle_device(c));
     const size_t nd = (size_t)c->n * (size_t)c->d * sizeof(float), db = (size_t)c->d * sizeof(float);
     if (e && c->E) {
         CU(cudaMemcpyAsync(c->E, e, nd, cudaMemcpyDeviceToDevice, c->stream));
@@ -600,6 +620,8 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
     const bool sign = c->compressor == COMPAMS_BLOCKSIGN;
     switch (which) {
         case COMPAMS_BUF_E:
+            if (c->compressed) return COMPAMS_ERR_INVALID_ARG;  // the residual is closed by compams_apply
+            RC(on_handle_device(c));
             RC(finish_residual(c));
             p = c->E;
             cnt = (int64_t)c->n * c->d;

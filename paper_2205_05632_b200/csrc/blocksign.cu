@@ -310,10 +310,10 @@ cudaError_t launch_bs_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
     if (c->chain) {  // small problem: the launch overlaps the tail of whatever kernel precedes it on the stream
         if (c->grad_bf16)
-            return launch_after(bs_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
-                                (const bf16_bits*)grads, c->e_is_x ? 1 : 0, c->segp);
-        return launch_after(bs_sweep_kernel<float>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
-                            (const float*)grads, c->e_is_x ? 1 : 0, c->segp);
+            return counted(c, launch_after(bs_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                                (const bf16_bits*)grads, c->e_is_x ? 1 : 0, c->segp));
+        return counted(c, launch_after(bs_sweep_kernel<float>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                            (const float*)grads, c->e_is_x ? 1 : 0, c->segp));
     }
     if (c->grad_bf16)
         bs_sweep_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads,
@@ -321,12 +321,12 @@ cudaError_t launch_bs_sweep(compams_context* c, const void* grads) {
     else
         bs_sweep_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const float*)grads,
                                                                  c->e_is_x ? 1 : 0, c->segp);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_bs_scales(compams_context* c) {
     dim3 grid((unsigned)c->M, (unsigned)c->n);
-    return launch_after(bs_scales_kernel, grid, dim3(kThreads), c->stream, c->tab, own_rows(c));
+    return counted(c, launch_after(bs_scales_kernel, grid, dim3(kThreads), c->stream, c->tab, own_rows(c)));
 }
 
 cudaError_t launch_bs_apply(compams_context* c, float* theta) {
@@ -335,18 +335,18 @@ cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     Tables t = c->tab;
     t.n = c->n_total;  // the average runs over every worker's message
     if (c->n == c->n_total)
-        return launch_after(bs_apply_kernel, dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), c->stream, t, b, theta,
-                            c->hp, c->segp);
+        return counted(c, launch_after(bs_apply_kernel, dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), c->stream, t, b, theta,
+                            c->hp, c->segp));
     // sharded workers: the other workers' messages were written by the caller's exchange, which is
     // ordered on the stream like any kernel; a plain launch waits for it
     bs_apply_kernel<<<dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_bs_materialize(compams_context* c) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
     bs_materialize_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->E, c->scales[c->scales_cur] + (size_t)c->row0 * (size_t)c->M);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 }  // namespace compams

@@ -20,6 +20,7 @@ constexpr int kBins1 = 2048;       // radix pass 1: key bits 30..20
 constexpr int kBins23 = 1024;      // radix passes 2, 3: key bits 19..10, 9..0
 constexpr int kBucketSpan = 1024;  // coordinates per server bucket: one CTA of the Top-k AMSGrad kernel
 constexpr int kMaxTimed = 4096;    // event pairs kept for per-kernel timing
+constexpr int64_t kMaxD = ((int64_t)1 << 31) - 4 * kTile;  // largest d: tile coordinates are 32-bit and overshoot a block's end
 
 constexpr uint32_t kNoPrediction = 0xffffffffu;  // tau_hat value that no key reaches
 constexpr int kTileCand = 1024;          // candidates one tile can stage in shared memory
@@ -136,7 +137,7 @@ struct compams_context {
     compams::BsBuffers bs{};
     compams::TopkBuffers tk{};
     int32_t* sel_small = nullptr;  // tiled blocks whose candidate lists one CTA selects from
-    int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists a cluster selects from
+    int32_t* sel_big = nullptr;    // tiled blocks whose candidate lists are cut into slices over many CTAs
     int n_sel_small = 0, n_sel_big = 0;
     int sel_parts = 1;  // slices a long candidate list is cut into
     std::vector<compams::SegState> seg_init_host;  // Top-k: the segments' state before the first step (set_state restores it)
@@ -149,6 +150,7 @@ struct compams_context {
     float* scales[2] = {nullptr, nullptr};
     int scales_cur = 0;
     bool e_is_x = false;  // Block-Sign: E holds the corrected gradient x of the last step, not e
+    bool compressed = false;  // compams_compress has run and its compams_apply has not: the step is half done
 
     // common device state
     float *E = nullptr, *m = nullptr, *v = nullptr, *vhat = nullptr, *gbar = nullptr;
@@ -172,7 +174,13 @@ struct compams_context {
 
 namespace compams {
 
-// Each launcher enqueues one kernel on ctx->stream and returns the launch status.
+// Adds a successfully enqueued kernel to the handle's launch count; passes the launch status through.
+inline cudaError_t counted(compams_context* c, cudaError_t e) {
+    if (e == cudaSuccess) ++c->launches;
+    return e;
+}
+
+// Each launcher enqueues its kernel(s) on ctx->stream and returns the launch status.
 cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, float* theta);
 cudaError_t launch_bs_sweep(compams_context* c, const void* grads);
 cudaError_t launch_bs_scales(compams_context* c);

@@ -175,12 +175,12 @@ cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, flo
             dense_mean_amsgrad_kernel<float, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
                                                                                   c->vhat, theta, c->hp);
     }
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_amsgrad(compams_context* c, float* theta) {
-    return launch_after(amsgrad_bucket_kernel, dim3((unsigned)c->tk.nbucket), dim3(kThreads), c->stream, c->d, c->tk, theta,
-                        c->hp);
+    return counted(c, launch_after(amsgrad_bucket_kernel, dim3((unsigned)c->tk.nbucket), dim3(kThreads), c->stream, c->d, c->tk, theta,
+                        c->hp));
 }
 
 }  // namespace compams

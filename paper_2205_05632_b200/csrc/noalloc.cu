@@ -36,7 +36,9 @@ static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_addr[kMaxDevices] = {nullptr};
 
-__global__ void __launch_bounds__(kThreads) bs_sweep_static_kernel(const float* __restrict__ G, float* __restrict__ X,
+// X is read and then overwritten by the same thread: it is read with plain loads (the read-only data path
+// is defined only for memory the kernel never writes) and carries no __restrict__.
+__global__ void __launch_bounds__(kThreads) bs_sweep_static_kernel(const float* __restrict__ G, float* X,
                                                                    const float* __restrict__ scales_prev,
                                                                    float* __restrict__ scales_out,
                                                                    uint32_t* __restrict__ bits, int64_t d,
@@ -58,12 +60,12 @@ __global__ void __launch_bounds__(kThreads) bs_sweep_static_kernel(const float* 
         const int64_t r = rw + it * 128 + lane * 4;
         float gv[4], xv[4];
         if (r + 3 < d) {
-            float4 a = load4_stream(g + r, cg), b = load4_stream(x + r, cx);
+            float4 a = load4_stream(g + r, cg), b = load4(x + r, cx);
             gv[0] = a.x; gv[1] = a.y; gv[2] = a.z; gv[3] = a.w;
             xv[0] = b.x; xv[1] = b.y; xv[2] = b.z; xv[3] = b.w;
         } else {
             for (int k = 0; k < 4; ++k) {
-                gv[k] = (r + k < d) ? g[r + k] : 0.0f;
+                gv[k] = (r + k < d) ? __ldg(g + r + k) : 0.0f;
                 xv[k] = (r + k < d) ? x[r + k] : 0.0f;
             }
         }

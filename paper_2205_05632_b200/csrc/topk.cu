@@ -1248,34 +1248,34 @@ cudaError_t launch_topk_small(compams_context* c, const void* grads) {
         topk_small_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads);
     else
         topk_small_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const float*)grads);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_topk_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
     if (c->chain) {
         if (c->grad_bf16)
-            return launch_after(topk_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
-                                (const bf16_bits*)grads, c->segp);
-        return launch_after(topk_sweep_kernel<float>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
-                            (const float*)grads, c->segp);
+            return counted(c, launch_after(topk_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                                (const bf16_bits*)grads, c->segp));
+        return counted(c, launch_after(topk_sweep_kernel<float>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
+                            (const float*)grads, c->segp));
     }
     if (c->grad_bf16)
         topk_sweep_kernel<bf16_bits><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const bf16_bits*)grads,
                                                                        c->segp);
     else
         topk_sweep_kernel<float><<<grid, kThreads, 0, c->stream>>>(c->tab, own_rows(c), (const float*)grads, c->segp);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 // On small problems the kernels of a step are launched as programmatic dependents of one another (each
 // waits for its predecessor before its first global access): the launch latency and the prologue of a
 // kernel then overlap the tail of the one before, which is most of what such a step costs.
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_chained(const compams_context* c, void (*kernel)(KArgs...), dim3 grid, dim3 block, Args... args) {
-    if (c->chain) return launch_after(kernel, grid, block, c->stream, args...);
+static cudaError_t launch_chained(compams_context* c, void (*kernel)(KArgs...), dim3 grid, dim3 block, Args... args) {
+    if (c->chain) return counted(c, launch_after(kernel, grid, block, c->stream, args...));
     kernel<<<grid, block, 0, c->stream>>>(static_cast<KArgs>(args)...);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_topk_select(compams_context* c) {
@@ -1303,15 +1303,15 @@ cudaError_t launch_topk_dense(compams_context* c) {
     }
     TopkBuffers b = own_rows(c);
     void* args[] = {(void*)&c->tab, (void*)&b};
-    return cudaLaunchCooperativeKernel((const void*)topk_dense_kernel, dim3((unsigned)c->dense_grid), dim3(kThreads), args,
-                                       0, c->stream);
+    return counted(c, cudaLaunchCooperativeKernel((const void*)topk_dense_kernel, dim3((unsigned)c->dense_grid),
+                                                  dim3(kThreads), args, 0, c->stream));
 }
 
 cudaError_t launch_topk_materialize(compams_context* c) {
     const int64_t words = c->tk.map_words;
     topk_materialize_kernel<<<(unsigned)((words + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
         (int64_t)c->n * c->d, c->tk.map_words, c->keptmap[c->map_cur], c->E);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_topk_scatter(compams_context* c) {
@@ -1320,9 +1320,9 @@ cudaError_t launch_topk_scatter(compams_context* c) {
     const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
     // (a sharded handle's exchange sits in front of this kernel: a plain launch waits for it)
     if (c->chain && c->n == c->n_total)
-        return launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count, c->row0);
+        return counted(c, launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count, c->row0));
     topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, c->row0);
-    return cudaGetLastError();
+    return counted(c, cudaGetLastError());
 }
 
 }  // namespace compams

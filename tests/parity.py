@@ -123,6 +123,11 @@ class Pair:
         if check_e:
             cnt["E"] = cnt.get("E", 0) + close(self.gpu.buffer("E"), self.cpu.buffer("E"), "E", s)
 
+    def set_lr(self, lr: float):
+        """eta_t of the following steps, on both sides (Algorithm 2 lets the learning rate vary with t)."""
+        self.gpu.set_lr(lr)
+        self.cpu.set_lr(lr)
+
     def close(self):
         self.gpu.close()
         self.cpu.close()

@@ -50,6 +50,10 @@ def test_invalid_arguments_are_rejected_before_any_cuda_call(lib):
     assert create(ctypes.byref(h), 2, 7, bad, 2, 1, 1.0, 1e-3, 0.9, 0.999, 1e-8) == -1     # empty block
     assert create(ctypes.byref(h), 2, 11, offs, 1, 1, 1.0, 1e-3, 0.9, 0.999, 1e-8) == -1   # last offset != d
     assert create(None, 2, 10, offs, 1, 1, 1.0, 1e-3, 0.9, 0.999, 1e-8) == -1
+    # d beyond what the 32-bit tile coordinates can address (they overshoot a block's end by up to two tiles)
+    big = (1 << 31) - 4 * 8192 + 1
+    offs_big = (ctypes.c_int64 * 2)(0, big)
+    assert create(ctypes.byref(h), 1, big, offs_big, 1, 1, 1.0, 1e-3, 0.9, 0.999, 1e-8) == -1
     assert not h.value
     assert lib.compams_destroy(None) == 0
     assert lib.compams_step(None, None, None) == -1

@@ -293,6 +293,30 @@ def test_amsgrad_vhat_holds_the_running_maximum():
 
 # ---------------------------------------------------------------- hand-worked traces of Algorithm 2
 
+def test_learning_rate_schedule_closed_form():
+    # Algorithm 2 with eta_t varying: a constant gradient g on one coordinate, k = d, one worker. Then
+    # m_t = (1 - b1^t) g, v_t = (1 - b2^t) g^2 (increasing, so vhat_t = v_t) and
+    # theta_{T+1} = theta_1 - sum_t eta_t m_t / sqrt(v_t + eps): every eta_t enters exactly one term, with
+    # that step's moments. A schedule applied one step late or early, or only the first eta, changes the sum.
+    b1, b2, eps, g = B1, B2, EPS, float(np.float32(0.37))  # the fp32 values the oracle computes with
+    etas = [float(np.float32(x)) for x in (1e-3, 1e-3, 1e-4, 5e-2, 1e-5, 2e-3)]
+    o = Oracle(1, 1, [0, 1], TOPK, 1.0, lr=etas[0], beta1=0.9, beta2=0.999, eps=1e-8)
+    theta = np.array([0.25], dtype=np.float32)
+    want = 0.25
+    for t, eta in enumerate(etas, start=1):
+        o.set_lr(eta)
+        o.step(np.array([[g]], dtype=np.float32), theta)
+        m = (1 - b1 ** t) * g
+        v = (1 - b2 ** t) * g * g
+        want -= eta * m / math.sqrt(v + eps)
+        assert abs(float(theta[0]) - want) <= 2e-6 * 0.25  # fp32 roundings of values up to theta_1 = 0.25
+    # the late and the early schedule are far outside that tolerance: the pin discriminates
+    late = 0.25 - sum(e * (1 - b1 ** t) * g / math.sqrt((1 - b2 ** t) * g * g + eps)
+                      for t, e in enumerate([etas[0]] + etas[:-1], start=1))
+    assert abs(late - want) > 1e-3
+    o.close()
+
+
 def read_trace(name):
     out = {}
     with open(os.path.join(GOLDEN, name)) as f:

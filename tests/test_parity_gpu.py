@@ -273,13 +273,13 @@ def test_config4_resnet50_shapes_layerwise(comp):
 @pytest.mark.parametrize("n", [1, 8, 32])
 def test_config5_sweep_points_oracle_sized(mode, n):
     from parity import run_workload
-    run_workload(W.sweep_point(1 << 20, n, mode, "cuda"), steps=3)
+    run_workload(W.sweep_point(1 << 20, n, mode, "cuda"), steps=10, check_e_every=3)
 
 
 @pytest.mark.parametrize("mode", ["topk", "sign", "dense"])
 def test_config5_sweep_point_d_2_24_n_8_against_the_full_oracle(mode):
     from parity import run_workload
-    run_workload(W.sweep_point(1 << 24, 8, mode, "cuda"), steps=3, check_e_every=3)
+    run_workload(W.sweep_point(1 << 24, 8, mode, "cuda"), steps=10, check_e_every=5)
 
 
 @pytest.mark.parametrize("mode", ["topk", "sign", "dense"])
@@ -372,18 +372,74 @@ def test_topk_layerwise_many_lists_single_cta_select():
     _pair_run(n, d, offs, TOPK, 0.03, _randn(n, d), steps=5, check_e_every=2)
 
 
-def test_set_lr_takes_effect_on_the_next_step():
-    d = 5000
-    opt = CompAMS(2, d, [0, d], BLOCKSIGN)
-    theta = torch.zeros(d, device="cuda")
-    G = torch.randn(2, d, device="cuda")
-    opt.step(G, theta)
-    moved = theta.clone()
-    assert moved.abs().max() > 0
-    opt.set_lr(0.0)
-    opt.step(G, theta)
-    assert torch.equal(theta, moved)
-    opt.close()
+@pytest.mark.parametrize("n", [3, 5])
+def test_topk_long_list_select_with_a_worker_count_that_is_not_a_power_of_two(n):
+    # one block long enough that its candidate list is cut into slices (two kernels over the slices); with
+    # n = 3 or 5 the mean over workers is an IEEE division, not a multiplication by 1 / n
+    d = 1_500_003
+    inexact = _pair_run(n, d, [0, d], TOPK, 0.01, _randn(n, d), steps=6, check_e_every=3)
+    assert inexact.get("gbar", 0) == 0
+
+
+@pytest.mark.parametrize("comp", [TOPK, BLOCKSIGN])
+def test_layerwise_over_more_than_two_hundred_large_blocks(comp):
+    # 230 blocks of 5,000 to 60,000 coordinates, n = 8: every block is tiled, the block list does not fit the
+    # kernel-argument copy (the per-tile table in global memory is used), and the selection runs over
+    # 8 x 230 candidate lists
+    sizes = [5000 + (7919 * b) % 55001 for b in range(230)]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    n, d = 8, offs[-1]
+    _pair_run(n, d, offs, comp, 0.01, _randn(n, d), steps=5, check_e_every=2)
+
+
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.02), (BLOCKSIGN, 1.0), (TOPK, 1.0)])
+def test_learning_rate_schedule_matches_the_oracle(comp, ratio):
+    # eta_t varies (Algorithm 2): divided by 10 in mid-run as in Section 5.1, then changed at every step;
+    # both sides are given the same eta_t before the same step
+    from parity import Pair
+    n, d = 3, 3 * 8192 + 517
+    gen = torch.Generator(device="cuda").manual_seed(21)
+    p = Pair(n, d, [0, 5000, d], comp, ratio, lr=1e-2)
+    schedule = [None, None, 1e-3, None, 1e-4, 3e-2, 0.0, 7e-3, 1e-3, 5e-4]
+    try:
+        p.start(0.1 * torch.randn(d, generator=gen, device="cuda"))
+        for t, lr in enumerate(schedule):
+            if lr is not None:
+                p.set_lr(lr)
+            before = p.theta_gpu.clone()
+            p.step(torch.randn(n, d, generator=gen, device="cuda"), check_e=(t % 3 == 0))
+            if lr == 0.0:
+                assert torch.equal(p.theta_gpu, before)  # eta_t = 0: the parameters rest, the moments move on
+    finally:
+        p.close()
+
+
+def test_calls_out_of_order_are_rejected():
+    # compress opens an iteration and apply closes it: in between the residual is not final, so the
+    # state cannot be read or replaced, and neither call may come twice in a row
+    n, d = 2, 3 * 8192
+    for comp, ratio in ((TOPK, 0.01), (BLOCKSIGN, 1.0)):
+        opt = CompAMS(n, d, [0, d], comp, ratio)
+        theta = torch.zeros(d, device="cuda")
+        G = torch.randn(n, d, device="cuda")
+        with pytest.raises(CompAMSError):
+            opt.apply(theta)                  # nothing compressed yet
+        opt.compress(G)
+        for call in (lambda: opt.compress(G), lambda: opt.step(G, theta), lambda: opt.buffer("E"),
+                     lambda: opt.get_state(), lambda: opt.set_state({"m": torch.zeros(d, device="cuda")})):
+            with pytest.raises(CompAMSError):
+                call()
+        opt.buffer("gbar")                    # buffers that the open iteration does not touch stay readable
+        opt.apply(theta)
+        opt.step(G, theta)                    # and the handle goes on as usual
+        assert opt.check_status() == 0
+        ref = CompAMS(n, d, [0, d], comp, ratio)
+        theta_ref = torch.zeros(d, device="cuda")
+        ref.step(G, theta_ref)
+        ref.step(G, theta_ref)
+        assert torch.equal(theta, theta_ref) and torch.equal(opt.buffer("E"), ref.buffer("E"))
+        opt.close()
+        ref.close()
 
 
 # ------------------------------------------------------------------ checkpoint / restore, traffic accounting
