@@ -16,6 +16,7 @@ from . import build as _build
 
 TOPK = 0
 BLOCKSIGN = 1
+RANDK = 2
 
 _lib = None
 
@@ -30,6 +31,14 @@ def lib() -> ctypes.CDLL:
                                     c.c_float, c.c_float, c.c_float, c.c_float]
         L.oracle_destroy.restype = None
         L.oracle_destroy.argtypes = [c.c_void_p]
+        L.oracle_philox4x64_10.restype = None
+        L.oracle_philox4x64_10.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
+        L.oracle_randk_permute.restype = c.c_uint64
+        L.oracle_randk_permute.argtypes = [c.c_uint64] * 6
+        L.oracle_randk_block.restype = None
+        L.oracle_randk_block.argtypes = [c.c_int64, c.c_int64, c.c_uint64, c.c_uint64, c.c_uint64, c.c_uint64, c.c_void_p]
+        L.oracle_set_seed.restype = None
+        L.oracle_set_seed.argtypes = [c.c_void_p, c.c_uint64, c.c_uint64]
         L.oracle_set_lr.restype = None
         L.oracle_set_lr.argtypes = [c.c_void_p, c.c_float]
         L.oracle_step.restype = c.c_int
@@ -76,6 +85,27 @@ def blocksign_scale(x) -> np.float32:
     return np.float32(lib().oracle_blocksign_scale(x.ctypes.data, x.size))
 
 
+def philox4x64_10(counter, key) -> np.ndarray:
+    """One block of Philox4x64-10: counter (4 uint64), key (2 uint64) -> 4 uint64."""
+    c = np.ascontiguousarray(counter, dtype=np.uint64)
+    k = np.ascontiguousarray(key, dtype=np.uint64)
+    out = np.zeros(4, dtype=np.uint64)
+    lib().oracle_philox4x64_10(c.ctypes.data, k.ctypes.data, out.ctypes.data)
+    return out
+
+
+def randk_permute(m: int, r: int, seed: int, step: int, worker: int, block: int) -> int:
+    """Image of r under the keyed permutation of {0..m-1} that Random-k draws its index sets from."""
+    return int(lib().oracle_randk_permute(int(m), int(r), int(seed), int(step), int(worker), int(block)))
+
+
+def randk_keep_mask(length: int, k: int, seed: int, step: int, worker: int, block: int) -> np.ndarray:
+    """Random-k on one block: boolean mask of the k kept coordinates for (seed, step, worker, block)."""
+    keep = np.zeros(int(length), dtype=np.uint8)
+    lib().oracle_randk_block(int(length), int(k), int(seed), int(step), int(worker), int(block), keep.ctypes.data)
+    return keep.astype(bool)
+
+
 def amsgrad(g, m, v, vhat, theta, lr, beta1, beta2, eps) -> None:
     """Algorithm 1 update, in place on the fp32 arrays m, v, vhat, theta."""
     for a in (g, m, v, vhat, theta):
@@ -116,6 +146,10 @@ class Oracle:
         rc = lib().oracle_step(self._h, G.ctypes.data, theta.ctypes.data)
         if rc != 0:
             raise RuntimeError("oracle_step failed")
+
+    def set_seed(self, seed: int, steps_done: int = 0) -> None:
+        """Random-k: the seed of the index sets and the number of iterations already done."""
+        lib().oracle_set_seed(self._h, int(seed), int(steps_done))
 
     def set_lr(self, lr: float) -> None:
         """eta_t of the following steps (Algorithm 2 lets the learning rate vary with t)."""

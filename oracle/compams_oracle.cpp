@@ -11,6 +11,11 @@
 // Reductions that the paper writes as exact sums (the block L1 norm of Definition 2, the average
 // over workers in Algorithm 2) are accumulated wider than fp32 and rounded once.
 //
+// Random-k (named among the deterministic sparsifiers in Section 2.1, not defined further) is this build's
+// reading, stated at randk_block below; its pins: the generator against an independent library
+// implementation, the index map being a bijection by brute force, set size, reproducibility and a
+// chi-square bound on the inclusion frequencies.
+//
 // Parity pins (tests/test_oracle_*.py): Top-k against brute force on tiny inputs; the error-feedback
 // identity C(x) + e_new = x (proof of Theorem 1); Block-Sign L1 preservation (Section 3.1); the
 // q-deviate bounds of Remark 1; the k = d and d_i = 1 identity cases (Assumption 1, q = 0);
@@ -32,7 +37,7 @@
 
 namespace {
 
-enum { COMPRESSOR_TOPK = 0, COMPRESSOR_BLOCKSIGN = 1 };
+enum { COMPRESSOR_TOPK = 0, COMPRESSOR_BLOCKSIGN = 1, COMPRESSOR_RANDK = 2 };
 
 inline uint32_t float_bits(float x) {
     uint32_t u;
@@ -93,6 +98,62 @@ float blocksign_scale(const float* x, int64_t len) {
     return (float)(S / (long double)len);
 }
 
+// Philox4x64-10, the counter-based generator of Salmon, Moraes, Dror and Shaw ("Parallel random numbers:
+// as easy as 1, 2, 3", SC 2011): a 256-bit counter and a 128-bit key give 256 pseudorandom bits. Ten
+// rounds; each multiplies two counter words by fixed odd constants, crosses the high and low halves
+// with the other two words and the key, and the key advances by Weyl constants between rounds.
+void philox4x64_10(const uint64_t ctr[4], const uint64_t key[2], uint64_t out[4]) {
+    const uint64_t M0 = 0xD2E7470EE14C6C93ull, M1 = 0xCA5A826395121157ull;
+    const uint64_t W0 = 0x9E3779B97F4A7C15ull, W1 = 0xBB67AE8584CAA73Bull;
+    uint64_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {
+            k0 += W0;
+            k1 += W1;
+        }
+        const unsigned __int128 p0 = (unsigned __int128)M0 * c0, p1 = (unsigned __int128)M1 * c2;
+        const uint64_t hi0 = (uint64_t)(p0 >> 64), lo0 = (uint64_t)p0, hi1 = (uint64_t)(p1 >> 64), lo1 = (uint64_t)p1;
+        const uint64_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// A keyed pseudorandom permutation of {0, ..., m-1}: a balanced Feistel network of four rounds over the
+// smallest even number of bits 2w with 2^(2w) >= m (at least 2), whose round function is the first word
+// of Philox4x64-10 at counter (right half, round, block, worker) under key (seed, step); a result
+// outside [0, m) is fed through the network again until it falls inside (cycle walking), which makes the
+// restriction to [0, m) a bijection.
+uint64_t randk_permute(uint64_t m, uint64_t r, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block) {
+    int bits = 2;
+    while (bits < 64 && ((uint64_t)1 << bits) < m) bits += 2;
+    const int w = bits / 2;
+    const uint64_t mask = ((uint64_t)1 << w) - 1;
+    const uint64_t key[2] = {seed, step};
+    uint64_t x = r;
+    do {
+        uint64_t L = x >> w, R = x & mask;
+        for (uint64_t round = 0; round < 4; ++round) {
+            const uint64_t ctr[4] = {R, round, block, worker};
+            uint64_t f[4];
+            philox4x64_10(ctr, key, f);
+            const uint64_t nR = L ^ (f[0] & mask);
+            L = R;
+            R = nR;
+        }
+        x = (L << w) | R;
+    } while (x >= m);
+    return x;
+}
+
+// Random-k on one block of `len` coordinates: the kept set is { pi(r) : r = 0 .. k-1 }, pi the permutation
+// above for this (seed, step, worker, block): k distinct coordinates, every k-subset (nearly) equally
+// likely, the same set whenever the four identifiers are the same. The values play no part.
+void randk_block(int64_t len, int64_t k, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block, uint8_t* keep) {
+    std::memset(keep, 0, (size_t)len);
+    for (int64_t r = 0; r < k; ++r) keep[randk_permute((uint64_t)len, (uint64_t)r, seed, step, worker, block)] = 1;
+}
+
 struct Oracle {
     int32_t n = 0;
     int64_t d = 0;
@@ -101,7 +162,9 @@ struct Oracle {
     int32_t compressor = 0;
     double k_ratio = 1.0;
     float lr = 0, beta1 = 0, beta2 = 0, eps = 0;
-    int64_t K = 0;                  // sum over blocks of kept_per_block (Top-k only)
+    uint64_t seed = 0;              // Random-k: the seed of the index sets
+    uint64_t steps_done = 0;        // iterations so far; the iteration being computed is steps_done + 1
+    int64_t K = 0;                  // sum over blocks of kept_per_block (Top-k and Random-k)
     std::vector<int64_t> seg_off;   // M + 1 prefix sums of kept_per_block
     // Algorithm 2 state
     std::vector<float> E;           // [n, d] error accumulators e_{t,i}
@@ -122,6 +185,17 @@ int64_t oracle_kept_per_block(double k_ratio, int64_t d_b) { return kept_per_blo
 void oracle_topk_block(const float* x, int64_t len, int64_t k, uint8_t* keep) { topk_block(x, len, k, keep); }
 
 float oracle_blocksign_scale(const float* x, int64_t len) { return blocksign_scale(x, len); }
+
+void oracle_philox4x64_10(const uint64_t* ctr, const uint64_t* key, uint64_t* out) { philox4x64_10(ctr, key, out); }
+
+uint64_t oracle_randk_permute(uint64_t m, uint64_t r, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block) {
+    return randk_permute(m, r, seed, step, worker, block);
+}
+
+void oracle_randk_block(int64_t len, int64_t k, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block,
+                        uint8_t* keep) {
+    randk_block(len, k, seed, step, worker, block, keep);
+}
 
 // Algorithm 1 / Algorithm 2 server update on d coordinates given the (averaged) gradient g:
 //   m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g^2;  vhat = max(vhat, v);
@@ -147,8 +221,8 @@ void oracle_amsgrad(int64_t d, const float* g, float* m, float* v, float* vhat, 
 void* oracle_create(int32_t n, int64_t d, const int64_t* block_offsets, int32_t num_blocks, int32_t compressor,
                     double k_ratio, float lr, float beta1, float beta2, float eps) {
     if (n < 1 || d < 1 || d >= ((int64_t)1 << 31) || num_blocks < 1 || !block_offsets) return nullptr;
-    if (compressor != COMPRESSOR_TOPK && compressor != COMPRESSOR_BLOCKSIGN) return nullptr;
-    if (compressor == COMPRESSOR_TOPK && !(k_ratio > 0.0 && k_ratio <= 1.0)) return nullptr;
+    if (compressor != COMPRESSOR_TOPK && compressor != COMPRESSOR_BLOCKSIGN && compressor != COMPRESSOR_RANDK) return nullptr;
+    if (compressor != COMPRESSOR_BLOCKSIGN && !(k_ratio > 0.0 && k_ratio <= 1.0)) return nullptr;
     if (block_offsets[0] != 0 || block_offsets[num_blocks] != d) return nullptr;
     for (int32_t b = 0; b < num_blocks; ++b)
         if (block_offsets[b + 1] <= block_offsets[b]) return nullptr;
@@ -165,7 +239,7 @@ void* oracle_create(int32_t n, int64_t d, const int64_t* block_offsets, int32_t 
     o->beta2 = beta2;
     o->eps = eps;
     o->seg_off.assign((size_t)num_blocks + 1, 0);
-    if (compressor == COMPRESSOR_TOPK)
+    if (compressor != COMPRESSOR_BLOCKSIGN)
         for (int32_t b = 0; b < num_blocks; ++b)
             o->seg_off[(size_t)b + 1] = o->seg_off[(size_t)b] + kept_per_block(k_ratio, o->off[b + 1] - o->off[b]);
     o->K = o->seg_off[(size_t)num_blocks];
@@ -183,6 +257,14 @@ void* oracle_create(int32_t n, int64_t d, const int64_t* block_offsets, int32_t 
 
 void oracle_destroy(void* h) { delete (Oracle*)h; }
 
+// Random-k: the seed of the index sets, and the number of iterations done so far (the next oracle_step is
+// iteration steps_done + 1; a run resumed from a checkpoint sets it to where the checkpoint was taken).
+void oracle_set_seed(void* h, uint64_t seed, uint64_t steps_done) {
+    if (!h) return;
+    ((Oracle*)h)->seed = seed;
+    ((Oracle*)h)->steps_done = steps_done;
+}
+
 // Algorithm 2 takes a learning rate eta_t per iteration: the value set here is the eta_t of every
 // following oracle_step until it is set again (Section 5.1 divides it by 10 at fixed epochs).
 void oracle_set_lr(void* h, float lr) {
@@ -197,6 +279,7 @@ int oracle_step(void* h, const float* G, float* theta) {
     const int32_t n = o->n;
     const int64_t d = o->d;
     const int32_t M = o->M;
+    const uint64_t t = ++o->steps_done;  // the iteration index, from 1
 
     // "parallel for worker i in [n]": the workers are independent until the server averages.
 #pragma omp parallel for schedule(dynamic, 1)
@@ -212,10 +295,13 @@ int oracle_step(void* h, const float* G, float* theta) {
         for (int32_t b = 0; b < M; ++b) {
             const int64_t lo = o->off[(size_t)b], len = o->off[(size_t)b + 1] - lo;
             const float* xb = x.data() + lo;
-            if (o->compressor == COMPRESSOR_TOPK) {
+            if (o->compressor == COMPRESSOR_TOPK || o->compressor == COMPRESSOR_RANDK) {
                 const int64_t k = o->seg_off[(size_t)b + 1] - o->seg_off[(size_t)b];
                 std::vector<uint8_t> keep((size_t)len);
-                topk_block(xb, len, k, keep.data());
+                if (o->compressor == COMPRESSOR_TOPK)
+                    topk_block(xb, len, k, keep.data());
+                else
+                    randk_block(len, k, o->seed, t, (uint64_t)i, (uint64_t)b, keep.data());
                 int32_t* out = o->kept_idx.data() + (size_t)i * (size_t)o->K + o->seg_off[(size_t)b];
                 int64_t r = 0;
                 for (int64_t j = 0; j < len; ++j) {

@@ -435,3 +435,101 @@ def test_lemma_bounds_and_monotone_vhat(comp):
         e2 = (o.buffer("E").astype(np.float64) ** 2).sum(axis=1).max()
         assert e2 <= 4 * q2 / (1 - q2) ** 2 * Gmax2                              # Lemma 2
         assert vh.max() <= 4 * (1 + q2) ** 3 / (1 - q2) ** 2 * Gmax2             # Lemma 4
+
+
+# ---------------------------------------------------------------- Random-k (Section 2.1 names it; the index rule is this build's reading)
+
+def test_philox4x64_matches_an_independent_library_implementation():
+    # numpy's Philox bit generator is Philox4x64-10; it advances its counter by one before it produces its
+    # first block, so its first four raw outputs are the block at counter + 1
+    rng = np.random.default_rng(31)
+    for _ in range(20):
+        ctr = [int(x) for x in rng.integers(0, 2 ** 63, size=4)]
+        key = [int(x) for x in rng.integers(0, 2 ** 63, size=2)]
+        want = np.random.Philox(counter=ctr, key=key).random_raw(4)
+        got = oracle.philox4x64_10([ctr[0] + 1] + ctr[1:], key)
+        assert np.array_equal(got, want)
+    # counter and key words all play a part: changing any one changes the block
+    base = oracle.philox4x64_10([1, 2, 3, 4], [5, 6])
+    for pos in range(4):
+        c = [1, 2, 3, 4]
+        c[pos] += 1
+        assert not np.array_equal(oracle.philox4x64_10(c, [5, 6]), base)
+    assert not np.array_equal(oracle.philox4x64_10([1, 2, 3, 4], [6, 6]), base)
+    assert not np.array_equal(oracle.philox4x64_10([1, 2, 3, 4], [5, 7]), base)
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4, 5, 7, 16, 17, 63, 64, 65, 100, 255, 256, 257, 1000, 4097])
+def test_randk_index_map_is_a_bijection(m):
+    for seed, step, worker, block in ((0, 1, 0, 0), (7, 3, 2, 5), (2 ** 40 + 1, 1000, 31, 160)):
+        image = sorted(oracle.randk_permute(m, r, seed, step, worker, block) for r in range(m))
+        assert image == list(range(m))
+
+
+def test_randk_sets_have_k_distinct_members_and_depend_on_every_identifier():
+    m, k = 5000, 50
+    base = oracle.randk_keep_mask(m, k, 3, 1, 0, 0)
+    assert base.sum() == k
+    assert np.array_equal(base, oracle.randk_keep_mask(m, k, 3, 1, 0, 0))  # same identifiers, same set
+    for other in ((4, 1, 0, 0), (3, 2, 0, 0), (3, 1, 1, 0), (3, 1, 0, 1)):
+        assert not np.array_equal(base, oracle.randk_keep_mask(m, k, *other))
+    # nested in k: the first k images of the permutation
+    assert np.all(oracle.randk_keep_mask(m, 20, 3, 1, 0, 0) <= base)
+    assert oracle.randk_keep_mask(m, m, 3, 1, 0, 0).all()
+
+
+def test_randk_inclusion_frequencies_are_uniform():
+    # over many steps every coordinate is kept about N k / m times: chi-square over the m coordinates against
+    # the hypergeometric variance N (k/m)(1 - k/m); 49 degrees of freedom put 99.99 % of the mass below 95.
+    # The first image pi(0) alone is uniform too.
+    m, k, N = 50, 5, 20000
+    counts = np.zeros(m)
+    first = np.zeros(m)
+    for step in range(1, N + 1):
+        counts += oracle.randk_keep_mask(m, k, 12345, step, 0, 0)
+        first[oracle.randk_permute(m, 0, 12345, step, 0, 0)] += 1
+    p = k / m
+    chi2 = float(((counts - N * p) ** 2).sum() / (N * p * (1 - p)))
+    assert chi2 < 95.0, chi2
+    chi2_first = float(((first - N / m) ** 2).sum() / (N / m))
+    assert chi2_first < 95.0, chi2_first
+    # pairs: coordinates 0 and 1 are kept together about N k (k-1) / (m (m-1)) times (no pairing by position)
+    both = sum(1 for step in range(1, 4001) if oracle.randk_keep_mask(m, k, 99, step, 0, 0)[:2].all())
+    expect = 4000 * k * (k - 1) / (m * (m - 1))
+    assert abs(both - expect) < 6 * math.sqrt(expect) + 1
+
+
+def test_randk_step_keeps_the_drawn_coordinates_and_conserves_the_error():
+    from oracle import RANDK
+    rng = np.random.default_rng(41)
+    offsets = [0, 64, 1000, 3000]
+    n, d, ratio, seed = 3, offsets[-1], 0.02, 77
+    o = Oracle(n, d, offsets, RANDK, ratio, **PAPER)
+    o.set_seed(seed)
+    theta = np.zeros(d, dtype=np.float32)
+    E_prev = np.zeros((n, d), dtype=np.float32)
+    for t in range(1, 5):
+        G = rng.standard_normal((n, d)).astype(np.float32)
+        o.step(G, theta)
+        X = G + E_prev
+        C, E = o.buffer("C").copy(), o.buffer("E").copy()
+        keep = np.zeros((n, d), dtype=bool)
+        for i in range(n):
+            for b in range(3):
+                lo, hi = offsets[b], offsets[b + 1]
+                keep[i, lo:hi] = oracle.randk_keep_mask(hi - lo, oracle.kept_per_block(ratio, hi - lo), seed, t, i, b)
+        assert np.array_equal(C, np.where(keep, X, np.float32(0)))          # g~ = x on the drawn set, 0 elsewhere
+        assert np.array_equal(E, np.where(keep, np.float32(0), X))          # e_{t+1} = x - g~
+        assert np.array_equal(o.buffer("kept_idx"), np.stack([np.flatnonzero(keep[i]) for i in range(n)]))
+        gbar = (C.astype(np.float64).sum(axis=0)).astype(np.float32) / np.float32(n)
+        assert np.array_equal(o.buffer("gbar"), gbar)
+        E_prev = E
+    o.close()
+    # k = d: every coordinate is drawn, the step is Algorithm 1 on the mean gradient
+    a = Oracle(2, 100, [0, 100], RANDK, 1.0, **PAPER)
+    b = Oracle(2, 100, [0, 100], TOPK, 1.0, **PAPER)
+    ta, tb = np.zeros(100, np.float32), np.zeros(100, np.float32)
+    G = rng.standard_normal((2, 100)).astype(np.float32)
+    a.step(G, ta)
+    b.step(G, tb)
+    assert np.array_equal(ta, tb) and not a.buffer("E").any()
