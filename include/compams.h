@@ -41,7 +41,9 @@ typedef struct compams_context* compams_handle;
 /* Compressors (Section 3.1). */
 enum compams_compressor {
     COMPAMS_TOPK = 0,      /* Definition 1, per block; k_b = clamp(floor(k_ratio * d_b), 1, d_b) */
-    COMPAMS_BLOCKSIGN = 1  /* Definition 2: sign(x_B) * ||x_B||_1 / d_B */
+    COMPAMS_BLOCKSIGN = 1, /* Definition 2: sign(x_B) * ||x_B||_1 / d_B */
+    COMPAMS_RANDK = 2      /* Random-k (Section 2.1 lists it beside Top-k): per block, k_b coordinates drawn uniformly
+                              at random whatever their values; see compams_set_seed for the drawing rule */
 };
 
 enum compams_status {
@@ -55,7 +57,8 @@ enum compams_status {
 
 /* Buffers readable through compams_get_buffer. */
 enum compams_buffer {
-    COMPAMS_BUF_E = 0,            /* float  [n, d]   error accumulators e_{t+1,i} (Algorithm 2, the residual update)          */
+    COMPAMS_BUF_E = 0,            /* float  [n, d]   error accumulators e_{t+1,i} (Algorithm 2, the residual update); not
+                                                    stored (count 0) when every k_b = d_b: they are identically zero */
     COMPAMS_BUF_M = 1,            /* float  [d]      first moment m_t                                            */
     COMPAMS_BUF_V = 2,            /* float  [d]      second moment v_t                                           */
     COMPAMS_BUF_VHAT = 3,         /* float  [d]      running maximum vhat_t                                      */
@@ -84,7 +87,8 @@ enum compams_kernel {
     COMPAMS_K_TOPK_DENSE = 5,         /* Top-k dense passes (one cooperative launch): radix histograms over x,
                                          threshold search, emission, lowest-index ties                        */
     COMPAMS_K_TOPK_MATERIALIZE = 6,   /* Top-k: zero e at the coordinates kept in the last step when E is read   */
-    /* 7, 8: reserved (never returned, never timed) */
+    COMPAMS_K_RANDK_EMIT = 7,         /* Random-k: every message slot computes its drawn coordinate and fetches x there */
+    /* 8: reserved (never returned, never timed) */
     COMPAMS_K_TOPK_SCATTER = 9,       /* Top-k: closes the step per segment; sparse scatter-accumulate         */
     COMPAMS_K_AMSGRAD = 10,           /* Top-k: AMSGrad update from the accumulated average                   */
     COMPAMS_K_TOPK_SMALL = 11,        /* Top-k: whole small blocks selected inside shared memory              */
@@ -104,8 +108,8 @@ enum compams_kernel {
  *   num_blocks     M >= 1. The compressor acts on each block separately (Section 3.1). With one
  *                  block Top-k is taken over the whole vector; with one block per tensor it is
  *                  layer-wise.
- *   compressor     COMPAMS_TOPK or COMPAMS_BLOCKSIGN.
- *   k_ratio        Top-k only, in (0, 1]: block b keeps k_b = max(1, min(d_b, floor(k_ratio * d_b)))
+ *   compressor     COMPAMS_TOPK, COMPAMS_BLOCKSIGN or COMPAMS_RANDK.
+ *   k_ratio        Top-k and Random-k, in (0, 1]: block b keeps k_b = max(1, min(d_b, floor(k_ratio * d_b)))
  *                  coordinates (Section 5.1 uses 0.01). If every k_b equals d_b the compressor is
  *                  the identity (q = 0 in Assumption 1): the step is then full-precision
  *                  distributed AMSGrad, e stays 0 and no (index, value) message is produced.
@@ -172,7 +176,11 @@ int compams_step_host(compams_handle h, const float* grads_host, float* theta_ho
  * on its own replica of theta, m, v, vhat: after the shards have exchanged their compressed gradients
  * (an all-gather of the message buffers - the only communication, and it is the caller's: this library
  * starts no collective), each applies the identical update, so the replicas stay bit-identical and
- * theta needs no broadcast.
+ * theta needs no broadcast. (The update is a function of the gathered messages alone. The one place where
+ * the order of arrival could show is the binary64 sum over workers at a coordinate, which is exact - hence
+ * order-free - while the magnitudes met at one coordinate lie within about 2^24 of one another at n = 32;
+ * beyond that spread the last bit of gbar may differ between replicas, and a job that must exclude even
+ * that re-broadcasts theta from one rank now and then.)
  *
  * compams_create_sharded - like compams_create, for a handle that holds workers first_worker ...
  *   first_worker + n_local - 1 of n_total (1 <= n_local, first_worker >= 0,
@@ -207,6 +215,31 @@ int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total
 int compams_compress(compams_handle h, const float* grads);
 int compams_apply(compams_handle h, float* theta);
 
+/*
+ * The handle's state in memory the caller allocates (for a harness that wants every device byte to come from
+ * its own allocator, e.g. one torch tensor): Algorithm 2's e, m, v, vhat, the message buffers and all scratch
+ * are cut from one region instead of being allocated one by one.
+ *
+ * compams_workspace_bytes - the size of that region for a handle with the given shape (the arguments mean
+ *   what they mean for compams_create_sharded; n_local == n_total for an unsharded handle). Host arithmetic
+ *   only: no CUDA call is made, no device is needed.
+ *   bytes   host; receives the size, a multiple of 256.
+ *
+ * compams_create_in_workspace - compams_create_sharded with the state placed in `workspace`.
+ *   workspace        device; at least workspace_bytes bytes, 256-byte aligned, on the current device. The caller
+ *                    keeps ownership: it must outlive the handle and is not freed by compams_destroy; its
+ *                    contents are the handle's while the handle lives.
+ *   workspace_bytes  its size; INVALID_ARG when smaller than compams_workspace_bytes reports.
+ *   No cudaMalloc is made for the state (small host-side objects - events for per-kernel timing - are still
+ *   created on demand, and compams_step_host allocates its staging buffers on first use).
+ */
+int compams_workspace_bytes(size_t* bytes, int32_t n_local, int32_t n_total, int64_t d, const int64_t* block_offsets,
+                            int32_t num_blocks, int32_t compressor, double k_ratio);
+int compams_create_in_workspace(compams_handle* out, void* workspace, size_t workspace_bytes, int32_t n_local,
+                                int32_t n_total, int32_t first_worker, int64_t d, const int64_t* block_offsets,
+                                int32_t num_blocks, int32_t compressor, double k_ratio, float lr, float beta1, float beta2,
+                                float eps);
+
 /* compams_destroy - free everything the handle owns (synchronises its stream first).
  * A null handle is a no-op. */
 int compams_destroy(compams_handle h);
@@ -214,6 +247,22 @@ int compams_destroy(compams_handle h);
 /* compams_set_stream - use `cuda_stream` (a cudaStream_t passed as void*, null = default stream)
  * for all later work of this handle. The caller orders earlier work against the new stream. */
 int compams_set_stream(compams_handle h, void* cuda_stream);
+
+/*
+ * compams_set_seed - Random-k: the seed of the index sets and the number of iterations already done (the
+ * next step is iteration iterations_done + 1; a new handle starts at seed 0, iterations_done 0; a run resumed
+ * from compams_set_state passes the iteration count of the checkpoint). Other compressors ignore both.
+ *
+ * The drawing rule (Section 2.1 only names Random-k; this is the library's reading, fixed so that a
+ * second implementation can reproduce the sets bit for bit): worker i keeps in block b, at iteration t,
+ * the coordinates block_offsets[b] + pi(r), r = 0 .. k_b - 1, where pi is a permutation of {0 .. d_b - 1}:
+ * a balanced Feistel network of four rounds over the smallest even number of bits 2w with 2^(2w) >= d_b
+ * (at least 2), applied again while the result is >= d_b. Round `round` maps (L, R) to (R, L xor (F & (2^w - 1)))
+ * with F the first output word of Philox4x64-10 (Salmon et al., SC 2011) at counter (R, round, b, i) under
+ * key (seed, t); the input is L = r >> w, R = r & (2^w - 1), the output (L << w) | R. Workers are numbered
+ * over the whole job (first_worker + local index on a sharded handle).
+ */
+int compams_set_seed(compams_handle h, uint64_t seed, uint64_t iterations_done);
 
 /* compams_set_lr - learning rate eta_t for the following steps (Algorithm 2 allows it to vary
  * with t; Section 5.2 divides it by 10 at fixed epochs). */

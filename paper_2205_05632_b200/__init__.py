@@ -5,9 +5,11 @@ no CPU fallback."""
 
 from .binding import (  # noqa: F401
     BLOCKSIGN,
+    RANDK,
     TOPK,
     CompAMS,
     CompAMSError,
     library_path,
     load_library,
+    workspace_bytes,
 )

@@ -15,6 +15,7 @@ import torch
 
 TOPK = 0
 BLOCKSIGN = 1
+RANDK = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_NAME = "libcompams.so"
@@ -32,7 +33,7 @@ _TYPESTR = {torch.float32: "<f4", torch.int32: "<i4", torch.int64: "<i8"}
 
 KERNELS = {
     "dense_mean_amsgrad": 0, "bs_sweep": 1, "bs_apply": 2, "bs_materialize": 3, "topk_sweep": 4, "topk_dense": 5,
-    "topk_materialize": 6, "topk_scatter": 9, "amsgrad": 10, "topk_small": 11,
+    "topk_materialize": 6, "randk_emit": 7, "topk_scatter": 9, "amsgrad": 10, "topk_small": 11,
     "topk_select": 12, "bs_scales": 13,
 }
 
@@ -75,6 +76,13 @@ def load_library() -> ctypes.CDLL:
     L.compams_create_sharded.restype = c.c_int
     L.compams_create_sharded.argtypes = [c.POINTER(H), c.c_int32, c.c_int32, c.c_int32, c.c_int64, c.POINTER(c.c_int64),
                                          c.c_int32, c.c_int32, c.c_double, c.c_float, c.c_float, c.c_float, c.c_float]
+    L.compams_workspace_bytes.restype = c.c_int
+    L.compams_workspace_bytes.argtypes = [c.POINTER(c.c_size_t), c.c_int32, c.c_int32, c.c_int64, c.POINTER(c.c_int64),
+                                          c.c_int32, c.c_int32, c.c_double]
+    L.compams_create_in_workspace.restype = c.c_int
+    L.compams_create_in_workspace.argtypes = [c.POINTER(H), c.c_void_p, c.c_size_t, c.c_int32, c.c_int32, c.c_int32,
+                                              c.c_int64, c.POINTER(c.c_int64), c.c_int32, c.c_int32, c.c_double,
+                                              c.c_float, c.c_float, c.c_float, c.c_float]
     L.compams_compress.restype = c.c_int
     L.compams_compress.argtypes = [H, c.c_void_p]
     L.compams_apply.restype = c.c_int
@@ -83,6 +91,8 @@ def load_library() -> ctypes.CDLL:
     L.compams_destroy.argtypes = [H]
     L.compams_set_stream.restype = c.c_int
     L.compams_set_stream.argtypes = [H, c.c_void_p]
+    L.compams_set_seed.restype = c.c_int
+    L.compams_set_seed.argtypes = [H, c.c_uint64, c.c_uint64]
     L.compams_set_lr.restype = c.c_int
     L.compams_set_lr.argtypes = [H, c.c_float]
     L.compams_get_state.restype = c.c_int
@@ -153,6 +163,18 @@ def blocksign_sweep_static_limits():
     return int(a.value), int(b.value)
 
 
+def workspace_bytes(n: int, d: int, block_offsets: Sequence[int], compressor: int, k_ratio: float = 1.0,
+                    n_total: Optional[int] = None) -> int:
+    """Bytes of device memory a CompAMS of this shape needs when its state lives in caller memory
+    (CompAMS(..., workspace=tensor)). Host arithmetic only: works without a GPU."""
+    offs = np.ascontiguousarray(block_offsets, dtype=np.int64)
+    out = ctypes.c_size_t(0)
+    _check(load_library().compams_workspace_bytes(ctypes.byref(out), int(n), int(n if n_total is None else n_total), int(d),
+                                                  offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), int(offs.size - 1),
+                                                  int(compressor), float(k_ratio)), "compams_workspace_bytes")
+    return int(out.value)
+
+
 class _DeviceView:
     """Exposes a raw device pointer to torch through the CUDA array interface."""
 
@@ -172,10 +194,13 @@ class CompAMS:
 
     def __init__(self, n: int, d: int, block_offsets: Sequence[int], compressor: int, k_ratio: float = 1.0,
                  lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 stream: Optional[torch.cuda.Stream] = None, n_total: Optional[int] = None, first_worker: int = 0):
+                 stream: Optional[torch.cuda.Stream] = None, n_total: Optional[int] = None, first_worker: int = 0,
+                 workspace: Optional[torch.Tensor] = None):
         """`n` workers live in this optimizer. With `n_total` > n they are workers `first_worker` ...
         `first_worker + n - 1` of a job whose other workers live in other optimizers (other GPUs): use
-        compress() / apply() with an exchange of the message buffers in between instead of step()."""
+        compress() / apply() with an exchange of the message buffers in between instead of step().
+        `workspace`: a contiguous CUDA uint8 tensor of at least workspace_bytes(...) bytes, 256-byte aligned,
+        that holds all of the optimizer's state (kept alive by this object); None: the library allocates."""
         self._L = load_library()
         self.n, self.d = int(n), int(d)
         self.n_total = self.n if n_total is None else int(n_total)
@@ -184,18 +209,28 @@ class CompAMS:
         self.M = int(offs.size - 1)
         self.compressor = int(compressor)
         self._h = ctypes.c_void_p()
-        rc = self._L.compams_create_sharded(ctypes.byref(self._h), self.n, self.n_total, self.first_worker, self.d,
-                                            offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), self.M,
-                                            self.compressor, float(k_ratio), float(lr), float(beta1), float(beta2),
-                                            float(eps))
+        self._workspace = workspace
+        shape = (self.n, self.n_total, self.first_worker, self.d, offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)),
+                 self.M, self.compressor, float(k_ratio), float(lr), float(beta1), float(beta2), float(eps))
+        if workspace is None:
+            rc = self._L.compams_create_sharded(ctypes.byref(self._h), *shape)
+        else:
+            if not (workspace.is_cuda and workspace.dtype == torch.uint8 and workspace.is_contiguous()):
+                raise CompAMSError("workspace must be a contiguous CUDA uint8 tensor")
+            rc = self._L.compams_create_in_workspace(ctypes.byref(self._h), ctypes.c_void_p(workspace.data_ptr()),
+                                                     int(workspace.numel()), *shape)
         if rc != 0:
             self._h = ctypes.c_void_p()
-        _check(rc, "compams_create_sharded")
+        _check(rc, "compams_create_sharded" if workspace is None else "compams_create_in_workspace")
         self.set_stream(stream if stream is not None else torch.cuda.current_stream())
 
     # -- calls ---------------------------------------------------------------------------------
     def set_stream(self, stream: torch.cuda.Stream) -> None:
         _check(self._L.compams_set_stream(self._h, ctypes.c_void_p(stream.cuda_stream)), "compams_set_stream")
+
+    def set_seed(self, seed: int, iterations_done: int = 0) -> None:
+        """Random-k: the seed of the index sets and the number of iterations already done."""
+        _check(self._L.compams_set_seed(self._h, int(seed), int(iterations_done)), "compams_set_seed")
 
     def set_lr(self, lr: float) -> None:
         _check(self._L.compams_set_lr(self._h, float(lr)), "compams_set_lr")
@@ -263,7 +298,7 @@ class CompAMS:
     def message_buffers(self):
         """The buffers an exchange between shards has to complete, as [n_total, width] views: every
         shard has filled rows first_worker ... first_worker + n - 1. Ask after compress()."""
-        names = ("topk_idx", "topk_val") if self.compressor == TOPK else ("sign_bits", "scales")
+        names = ("topk_idx", "topk_val") if self.compressor in (TOPK, RANDK) else ("sign_bits", "scales")
         return [self.buffer(name) for name in names]
 
     def step_host(self, grads: torch.Tensor, theta: torch.Tensor) -> None:
@@ -287,6 +322,8 @@ class CompAMS:
                "compams_get_buffer")
         dt = _BUFFER_DTYPES[name]
         if cnt.value == 0 or not ptr.value:
+            if name == "E":  # every k_b = d_b: the error accumulators are identically zero and not stored
+                return torch.zeros(self.n, self.d, dtype=dt, device="cuda")
             return torch.empty(0, dtype=dt, device="cuda")
         t = torch.as_tensor(_DeviceView(ptr.value, cnt.value, dt, self), device="cuda")
         if name == "E":

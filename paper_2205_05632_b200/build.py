@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcompams.so")
-SOURCES = ["api.cu", "dense.cu", "blocksign.cu", "topk.cu", "noalloc.cu"]
-HEADERS = ["common.cuh", "context.h", os.path.join("..", "..", "include", "compams.h")]
+SOURCES = ["api.cu", "dense.cu", "blocksign.cu", "topk.cu", "randk.cu", "noalloc.cu"]
+HEADERS = ["common.cuh", "context.h", "scatter.cuh", os.path.join("..", "..", "include", "compams.h")]
 
 # -fmad=false: no fused multiply-add anywhere, so each fp32 operation of the update rounds on its own.
 NVCC_FLAGS = [

@@ -30,6 +30,16 @@ template <typename T>
 int dev_alloc(compams_context* c, T** out, size_t count, bool zero = true) {
     *out = nullptr;
     if (count == 0) count = 1;
+    if (c->plan_only || c->ws) {
+        // buffers are cut from one region, each on a 256-byte boundary
+        const size_t off = (c->ws_used + 255) & ~(size_t)255;
+        c->ws_used = off + count * sizeof(T);
+        if (c->plan_only) return COMPAMS_OK;
+        if (c->ws_used > c->ws_bytes) return COMPAMS_ERR_INVALID_ARG;  // the caller's region is too small
+        if (zero) CU(cudaMemsetAsync(c->ws + off, 0, count * sizeof(T), c->stream));
+        *out = (T*)(c->ws + off);
+        return COMPAMS_OK;
+    }
     void* p = nullptr;
     cudaError_t e = cudaMalloc(&p, count * sizeof(T));
     if (e != cudaSuccess) {
@@ -47,7 +57,7 @@ template <typename T>
 int dev_upload(compams_context* c, T** out, const std::vector<T>& host) {
     int rc = dev_alloc(c, out, host.size(), false);
     if (rc) return rc;
-    if (!host.empty()) CU(cudaMemcpy(*out, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice));
+    if (!host.empty() && !c->plan_only) CU(cudaMemcpy(*out, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice));
     return COMPAMS_OK;
 }
 
@@ -99,7 +109,7 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
             si.slot0 = c->seg_off[(size_t)b];
             si.kb = (uint32_t)kb;
             // the candidate path pays off for sparse selections only: at most 1/32 of the block kept
-            int64_t cap = (kb * 32 <= len) ? 8 * kb + 1024 : 0;
+            int64_t cap = (!c->randk && kb * 32 <= len) ? 8 * kb + 1024 : 0;
             if (cap > len) cap = len;
             si.cap = (uint32_t)cap;
             si.cand_off = cand_total;
@@ -175,8 +185,10 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
 }
 
 int init_context(compams_context* c, const int64_t* block_offsets) {
-    CU(cudaGetDevice(&c->device));
-    CU(cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device));
+    if (!c->plan_only) {
+        CU(cudaGetDevice(&c->device));
+        CU(cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device));
+    }
     const int32_t n = c->n, M = c->M;
     const int64_t d = c->d;
     c->off.assign(block_offsets, block_offsets + M + 1);
@@ -192,7 +204,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
     RC(dev_alloc(c, &c->gbar, (size_t)d));
     RC(dev_alloc(c, &c->status, 8));
 
-    if (c->compressor == COMPAMS_TOPK) {
+    if (c->sparse()) {
         c->seg_off.assign((size_t)M + 1, 0);
         bool identity = true;
         for (int32_t b = 0; b < M; ++b) {
@@ -205,14 +217,15 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         c->K = identity ? 0 : c->seg_off[(size_t)M];
     }
 
-    if (c->compressor == COMPAMS_TOPK && c->identity) {
-        // full-precision distributed AMSGrad: e is identically zero, kept only so that BUF_E can be read
-        RC(dev_alloc(c, &c->E, (size_t)n * (size_t)d));
-    } else if (c->compressor == COMPAMS_TOPK) {
+    if (c->sparse() && c->identity) {
+        // full-precision distributed AMSGrad: e is identically zero and not stored
+    } else if (c->sparse()) {
         RC(dev_alloc(c, &c->E, (size_t)n * (size_t)d));
         RC(dev_upload(c, &c->d_seg_off, c->seg_off));
         std::vector<int32_t> small, large;
-        for (int32_t b = 0; b < M; ++b) ((c->off[b + 1] - c->off[b] <= kSmallMax) ? small : large).push_back(b);
+        // (Random-k has no selection: every block is tiled for the sweep, none goes to the shared-memory select)
+        for (int32_t b = 0; b < M; ++b)
+            ((!c->randk && c->off[b + 1] - c->off[b] <= kSmallMax) ? small : large).push_back(b);
         RC(build_tiles(c, large, true));
         TopkBuffers& t = c->tk;
         t.E = c->E;
@@ -226,7 +239,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         // rows are filled by the caller's exchange before compams_apply
         RC(dev_alloc(c, &t.idx, (size_t)c->n_total * (size_t)c->K));
         RC(dev_alloc(c, &t.val, (size_t)c->n_total * (size_t)c->K));
-        RC(dev_alloc(c, &t.hist, (size_t)n * (size_t)c->tab.nseg * kBins1));
+        RC(dev_alloc(c, &t.hist, c->randk ? 1 : (size_t)n * (size_t)c->tab.nseg * kBins1));
         {
             SegState init{};
             init.tau_hat = kNoPrediction;
@@ -242,7 +255,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
             std::vector<uint32_t> dc(1, never * (uint32_t)n);
             RC(dev_upload(c, &t.dense_count, dc));
         }
-        RC(dev_alloc(c, &t.tile_ties, (size_t)n * (size_t)c->tab.ntiles));
+        RC(dev_alloc(c, &t.tile_ties, c->randk ? 1 : (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &t.cand, (size_t)n * (size_t)t.cand_total, false));
         RC(dev_alloc(c, &t.acc, (size_t)d));
         t.map_words = ((int64_t)n * d + 31) / 32;
@@ -292,7 +305,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         s.v = c->v;
         s.vhat = c->vhat;
     }
-    CU(cudaDeviceSynchronize());
+    if (!c->plan_only) CU(cudaDeviceSynchronize());
     return COMPAMS_OK;
 }
 
@@ -334,6 +347,7 @@ int run_kernel(compams_context* c, int kernel, F&& launch) {
 // compression, the residual; the compressed gradients land in this handle's rows of the message buffers.
 int compress_device(compams_context* c, const void* grads) {
     ++c->steps_done;
+    ++c->iter;
     if (c->compressor == COMPAMS_BLOCKSIGN) {
         c->scales_cur ^= 1;
         RC(run_kernel(c, COMPAMS_K_BS_SWEEP, [&] { return launch_bs_sweep(c, grads); }));
@@ -347,6 +361,16 @@ int compress_device(compams_context* c, const void* grads) {
     c->tk.kept_cur = c->keptmap[c->map_cur];
     c->tk.kept_prev = c->e_mask_pending ? c->keptmap[c->map_cur ^ 1] : nullptr;
     CU(cudaMemsetAsync(c->tk.kept_cur, 0, (size_t)c->tk.map_words * sizeof(uint32_t), c->stream));
+    if (c->randk) {
+        // no selection: the sweep leaves x in E, then every message slot fetches the x of its drawn coordinate;
+        // with all workers in this handle the pairs go to the server in the same kernel, otherwise
+        // compams_apply delivers the exchanged messages
+        const bool deliver = c->n == c->n_total;
+        RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
+        RC(run_kernel(c, COMPAMS_K_RANDK_EMIT, [&] { return launch_randk_emit(c, deliver); }));
+        if (deliver) c->e_mask_pending = true;
+        return COMPAMS_OK;
+    }
     if (c->tk.nsmall > 0) RC(run_kernel(c, COMPAMS_K_TOPK_SMALL, [&] { return launch_topk_small(c, grads); }));
     if (c->tab.ntiles > 0) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
@@ -361,30 +385,38 @@ int apply_device(compams_context* c, float* theta) {
     if (c->compressor == COMPAMS_BLOCKSIGN) {
         return run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); });
     }
-    RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c); }));
-    c->e_mask_pending = true;
+    // (a Random-k step with every worker in this handle has delivered its messages already)
+    if (!(c->randk && c->n == c->n_total)) {
+        RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c, !c->randk); }));
+        c->e_mask_pending = true;
+    }
     RC(run_kernel(c, COMPAMS_K_AMSGRAD, [&] { return launch_amsgrad(c, theta); }));
     return COMPAMS_OK;
 }
 
 int step_device(compams_context* c, const void* grads, float* theta) {
-    if (c->compressor == COMPAMS_TOPK && c->identity) {
+    if (c->sparse() && c->identity) {
         ++c->steps_done;
+        ++c->iter;
         return run_kernel(c, COMPAMS_K_DENSE_MEAN_AMSGRAD, [&] { return launch_dense_mean_amsgrad(c, grads, theta); });
     }
     RC(compress_device(c, grads));
     return apply_device(c, theta);
 }
 
+// `ws` null: every buffer is the library's own allocation. `ws` non-null: the buffers are cut from the caller's
+// region of `ws_bytes` bytes. `plan` non-null: nothing is created; *plan receives the bytes such a region needs.
 int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0, int64_t d, const int64_t* block_offsets,
-                  int32_t num_blocks, int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps) {
-    if (!out || !block_offsets) return COMPAMS_ERR_INVALID_ARG;
+                  int32_t num_blocks, int32_t compressor, double k_ratio, float lr, float beta1, float beta2, float eps,
+                  void* ws = nullptr, size_t ws_bytes = 0, size_t* plan = nullptr) {
+    if ((!out && !plan) || !block_offsets) return COMPAMS_ERR_INVALID_ARG;
     // the tiled kernels address a block with 32-bit coordinates that may run up to two tiles past its end
     if (n < 1 || n_total > 65535 || row0 < 0 || (int64_t)row0 + n > n_total || d < 1 || d > kMaxD ||
         num_blocks < 1 || (int64_t)num_blocks > d)
         return COMPAMS_ERR_INVALID_ARG;
-    if (compressor != COMPAMS_TOPK && compressor != COMPAMS_BLOCKSIGN) return COMPAMS_ERR_INVALID_ARG;
-    if (compressor == COMPAMS_TOPK && !(k_ratio > 0.0 && k_ratio <= 1.0)) return COMPAMS_ERR_INVALID_ARG;
+    if (compressor != COMPAMS_TOPK && compressor != COMPAMS_BLOCKSIGN && compressor != COMPAMS_RANDK)
+        return COMPAMS_ERR_INVALID_ARG;
+    if (compressor != COMPAMS_BLOCKSIGN && !(k_ratio > 0.0 && k_ratio <= 1.0)) return COMPAMS_ERR_INVALID_ARG;
     if (!(lr == lr) || !(beta1 == beta1) || !(beta2 == beta2) || !(eps == eps)) return COMPAMS_ERR_INVALID_ARG;
     if (block_offsets[0] != 0 || block_offsets[num_blocks] != d) return COMPAMS_ERR_INVALID_ARG;
     for (int32_t b = 0; b < num_blocks; ++b)
@@ -398,7 +430,8 @@ int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0,
     c->d = d;
     c->M = num_blocks;
     c->compressor = compressor;
-    c->k_ratio = (compressor == COMPAMS_TOPK) ? k_ratio : 1.0;
+    c->k_ratio = (compressor != COMPAMS_BLOCKSIGN) ? k_ratio : 1.0;
+    c->randk = compressor == COMPAMS_RANDK;
     c->hp.lr = lr;
     c->hp.beta1 = beta1;
     c->hp.beta2 = beta2;
@@ -408,6 +441,9 @@ int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0,
     c->chain = (int64_t)n * d <= kChainMaxElems;
     c->hp.nf = (float)n_total;
     c->hp.inv_nf = ((n_total & (n_total - 1)) == 0) ? 1.0f / (float)n_total : 0.0f;
+    c->plan_only = plan != nullptr;
+    c->ws = (unsigned char*)ws;
+    c->ws_bytes = ws_bytes;
     int rc;
     try {
         rc = init_context(c, block_offsets);
@@ -416,7 +452,8 @@ int create_handle(compams_handle* out, int32_t n, int32_t n_total, int32_t row0,
     }
     // sharded workers exchange compressed gradients; the uncompressed mode (k = d) has none to exchange
     if (!rc && n != n_total && c->identity) rc = COMPAMS_ERR_INVALID_ARG;
-    if (rc) {
+    if (rc || plan) {
+        if (!rc) *plan = (c->ws_used + 255) & ~(size_t)255;
         free_context(c);
         return rc;
     }
@@ -440,9 +477,25 @@ int compams_create_sharded(compams_handle* out, int32_t n_local, int32_t n_total
                          beta2, eps);
 }
 
+int compams_workspace_bytes(size_t* bytes, int32_t n_local, int32_t n_total, int64_t d, const int64_t* block_offsets,
+                            int32_t num_blocks, int32_t compressor, double k_ratio) {
+    if (!bytes) return COMPAMS_ERR_INVALID_ARG;
+    return create_handle(nullptr, n_local, n_total, 0, d, block_offsets, num_blocks, compressor, k_ratio, 0.0f, 0.0f, 0.0f,
+                         0.0f, nullptr, 0, bytes);
+}
+
+int compams_create_in_workspace(compams_handle* out, void* workspace, size_t workspace_bytes, int32_t n_local,
+                                int32_t n_total, int32_t first_worker, int64_t d, const int64_t* block_offsets,
+                                int32_t num_blocks, int32_t compressor, double k_ratio, float lr, float beta1, float beta2,
+                                float eps) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return COMPAMS_ERR_INVALID_ARG;
+    return create_handle(out, n_local, n_total, first_worker, d, block_offsets, num_blocks, compressor, k_ratio, lr, beta1,
+                         beta2, eps, workspace, workspace_bytes);
+}
+
 static int compress_any(compams_handle c, const void* grads, bool bf16) {
     if (!c || !grads || (reinterpret_cast<uintptr_t>(grads) & (bf16 ? 1u : 3u))) return COMPAMS_ERR_INVALID_ARG;
-    if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;  // k = d: nothing is compressed
+    if (c->sparse() && c->identity) return COMPAMS_ERR_INVALID_ARG;  // k = d: nothing is compressed
     if (c->compressed) return COMPAMS_ERR_INVALID_ARG;  // the previous compress has not been applied yet
     RC(on_handle_device(c));
     c->grad_bf16 = bf16;
@@ -461,7 +514,7 @@ int compams_compress_bf16(compams_handle c, const void* grads_bf16) { return com
 
 int compams_apply(compams_handle c, float* theta) {
     if (!c || !theta || (reinterpret_cast<uintptr_t>(theta) & 15u)) return COMPAMS_ERR_INVALID_ARG;
-    if (c->compressor == COMPAMS_TOPK && c->identity) return COMPAMS_ERR_INVALID_ARG;
+    if (c->sparse() && c->identity) return COMPAMS_ERR_INVALID_ARG;
     if (!c->compressed) return COMPAMS_ERR_INVALID_ARG;  // nothing to apply: compams_compress comes first
     RC(on_handle_device(c));
     c->compressed = false;
@@ -537,6 +590,13 @@ int compams_set_stream(compams_handle c, void* cuda_stream) {
     return COMPAMS_OK;
 }
 
+int compams_set_seed(compams_handle c, uint64_t seed, uint64_t iterations_done) {
+    if (!c || c->compressed) return COMPAMS_ERR_INVALID_ARG;
+    c->seed = seed;
+    c->iter = iterations_done;
+    return COMPAMS_OK;
+}
+
 int compams_set_lr(compams_handle c, float lr) {
     if (!c || !(lr == lr)) return COMPAMS_ERR_INVALID_ARG;
     c->hp.lr = lr;
@@ -545,7 +605,7 @@ int compams_set_lr(compams_handle c, float lr) {
 
 // Finishes the residual update where it has been deferred, so that E holds e.
 static int finish_residual(compams_context* c) {
-    if (c->compressor == COMPAMS_TOPK && !c->identity && c->e_mask_pending) {
+    if (c->sparse() && !c->identity && c->e_mask_pending) {
         RC(run_kernel(c, COMPAMS_K_TOPK_MATERIALIZE, [&] { return launch_topk_materialize(c); }));
         c->e_mask_pending = false;
     }
@@ -616,11 +676,12 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
     if (!c || !dev_ptr || !count) return COMPAMS_ERR_INVALID_ARG;
     void* p = nullptr;
     int64_t cnt = 0;
-    const bool topk = c->compressor == COMPAMS_TOPK && !c->identity;
+    const bool topk = c->sparse() && !c->identity;
     const bool sign = c->compressor == COMPAMS_BLOCKSIGN;
     switch (which) {
         case COMPAMS_BUF_E:
             if (c->compressed) return COMPAMS_ERR_INVALID_ARG;  // the residual is closed by compams_apply
+            if (!c->E) break;  // every k_b = d_b: e is identically zero and not stored
             RC(on_handle_device(c));
             RC(finish_residual(c));
             p = c->E;
@@ -695,7 +756,7 @@ const char* compams_error_string(int status) {
 const char* compams_kernel_name(int32_t kernel) {
     static const char* names[COMPAMS_K_COUNT] = {
         "dense_mean_amsgrad", "bs_sweep", "bs_apply", "bs_materialize", "topk_sweep", "topk_dense",
-        "topk_materialize", "unused", "unused", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
+        "topk_materialize", "randk_emit", "reserved", "topk_scatter", "amsgrad", "topk_small", "topk_select", "bs_scales"};
     return (kernel >= 0 && kernel < COMPAMS_K_COUNT) ? names[kernel] : "unknown";
 }
 

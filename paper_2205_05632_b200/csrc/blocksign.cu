@@ -111,8 +111,11 @@ __device__ __forceinline__ void bs_sweep_tile(const GT* __restrict__ g, float* _
 // sign words stay indexed by coordinate: word q of the block takes its low 32 - s bits from the
 // q-th group of 32 shifted coordinates and its high s bits from the next group. The word a tile
 // shares with the next tile is put together by bs_scales from the two shares left in `edge`.
+#ifndef COMPAMS_BF16_SWEEP_CTAS
+#define COMPAMS_BF16_SWEEP_CTAS 8
+#endif
 template <typename GT>
-__global__ void __launch_bounds__(kThreads, 8) bs_sweep_kernel(Tables t, BsBuffers b, const GT* __restrict__ G,
+__global__ void __launch_bounds__(kThreads, sizeof(GT) == 2 ? COMPAMS_BF16_SWEEP_CTAS : 8) bs_sweep_kernel(Tables t, BsBuffers b, const GT* __restrict__ G,
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     __shared__ uint32_t sh_first[kWarps];
@@ -334,12 +337,12 @@ cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     b.scales_cur = c->scales[c->scales_cur];
     Tables t = c->tab;
     t.n = c->n_total;  // the average runs over every worker's message
+    const dim3 grid((unsigned)c->tab.ntiles * kWarps);
     if (c->n == c->n_total)
-        return counted(c, launch_after(bs_apply_kernel, dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), c->stream, t, b, theta,
-                            c->hp, c->segp));
+        return counted(c, launch_after(bs_apply_kernel, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp));
     // sharded workers: the other workers' messages were written by the caller's exchange, which is
     // ordered on the stream like any kernel; a plain launch waits for it
-    bs_apply_kernel<<<dim3((unsigned)c->tab.ntiles * kWarps), dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
+    bs_apply_kernel<<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
     return counted(c, cudaGetLastError());
 }
 

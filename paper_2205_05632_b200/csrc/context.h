@@ -50,7 +50,8 @@ struct SegState {
     uint32_t need_order;  // 1 when ties_take < ties_total: the lowest indices must be chosen
     uint32_t emit_count;  // message slots handed out so far
     uint32_t sel_ready;   // multi-CTA select: the threshold bin has been found, the emit kernel may run
-    uint32_t pad[2];
+    uint32_t boost;       // the candidate margin is doubled this many times (raised when a list came up short)
+    uint32_t streak;      // selections decided inside the list since the margin last changed
 };
 
 // Block / tile tables shared by the tiled kernels (device pointers).
@@ -121,7 +122,11 @@ struct compams_context {
     int32_t M = 0;
     int32_t compressor = 0;
     double k_ratio = 1.0;
-    bool identity = false;     // Top-k with every k_b == d_b
+    bool identity = false;     // Top-k or Random-k with every k_b == d_b
+    bool randk = false;        // Random-k: the kept sets are drawn, not selected
+    uint64_t seed = 0;         // Random-k: seed of the index sets
+    uint64_t iter = 0;         // iterations so far (Random-k keys its sets by the iteration index, from 1)
+    bool sparse() const { return compressor != COMPAMS_BLOCKSIGN; }  // Top-k or Random-k: (index, value) messages
     compams::HyperParams hp{};
     cudaStream_t stream = nullptr;
     int num_sms = 148;
@@ -152,13 +157,18 @@ struct compams_context {
     bool e_is_x = false;  // Block-Sign: E holds the corrected gradient x of the last step, not e
     bool compressed = false;  // compams_compress has run and its compams_apply has not: the step is half done
 
+
     // common device state
     float *E = nullptr, *m = nullptr, *v = nullptr, *vhat = nullptr, *gbar = nullptr;
     uint32_t* status = nullptr;
     int64_t* d_off = nullptr;
     int64_t* d_seg_off = nullptr;
     int64_t* d_word_off = nullptr;
-    std::vector<void*> owned;  // every device allocation, for destroy
+    std::vector<void*> owned;  // every device allocation of the library's own, for destroy
+    // state placed in caller memory (compams_create_in_workspace), or only sized (compams_workspace_bytes)
+    bool plan_only = false;          // nothing is allocated or touched: the buffers are only added up
+    unsigned char* ws = nullptr;     // caller's device memory the buffers are cut from (null: cudaMalloc each)
+    size_t ws_bytes = 0, ws_used = 0;
 
     // staging for compams_step_host
     float* stage_grads = nullptr;
@@ -191,7 +201,8 @@ cudaError_t launch_topk_sweep(compams_context* c, const void* grads);
 cudaError_t launch_topk_select(compams_context* c);
 cudaError_t launch_topk_dense(compams_context* c);
 cudaError_t launch_topk_materialize(compams_context* c);
-cudaError_t launch_topk_scatter(compams_context* c);
+cudaError_t launch_topk_scatter(compams_context* c, bool close);
+cudaError_t launch_randk_emit(compams_context* c, bool deliver);
 cudaError_t launch_amsgrad(compams_context* c, float* theta);
 
 }  // namespace compams

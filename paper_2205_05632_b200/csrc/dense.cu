@@ -69,9 +69,14 @@ __global__ void __launch_bounds__(kThreads, CTAS_PER_SM) dense_mean_amsgrad_kern
 }
 
 // Server update of the Top-k path, one CTA per bucket of kBucketSpan coordinates: the bucket's kept
-// entries (all workers) are summed in binary64 in shared memory - exact, hence independent of the
-// order - then gbar = (float)sum / n and Algorithm 2, the moment, maximum and parameter updates. Entries that did not fit their
-// bucket were added to acc[] by the scatter kernel and are folded in (and acc cleared) here.
+// entries (all workers) are summed in binary64 in shared memory, in the order the atomics arrive, then
+// gbar = (float)sum / n and Algorithm 2, the moment, maximum and parameter updates. The binary64 sum of the
+// fp32 terms of one coordinate is exact - and then the order cannot matter - as long as 24 + (the spread of
+// the terms' exponents) + log2 n <= 53, i.e. the magnitudes kept at one coordinate lie within 2^24 of one
+// another at n = 32. Wider spreads (one worker keeps 1e-12 where another keeps 1) can round differently from
+// run to run in the last bit of gbar, which stays inside the tolerance the step is specified to. Entries
+// that did not fit their bucket were added to acc[] by the scatter kernel and are folded in (and acc
+// cleared) here.
 __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, TopkBuffers b, float* __restrict__ theta,
                                                                      HyperParams hp) {
     static_assert(kBucketSpan == 4 * kThreads, "one float4 group per thread");

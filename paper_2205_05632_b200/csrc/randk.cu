@@ -1,0 +1,95 @@
+// Random-k path of the COMP-AMS step: every (worker, block) keeps k_b coordinates drawn uniformly at random,
+// whatever their values (Section 2.1 lists Random-k beside Top-k among the deterministic sparsifiers; with
+// error feedback the dropped coordinates wait in e until they are drawn).
+//
+// The kept set of (step t, worker i, block b) is { pi(r) : r = 0 .. k_b - 1 }, pi a keyed pseudorandom
+// permutation of the block's coordinates: a balanced Feistel network of four rounds over the smallest even
+// number of bits that covers d_b, with cycle walking back into [0, d_b); the round function is the first
+// word of Philox4x64-10 (Salmon, Moraes, Dror, Shaw, SC 2011) at counter (right half, round, b, i) under
+// key (seed, t). Being the image of k_b distinct inputs under a bijection, the set has exactly k_b members
+// and needs no selection pass: the sweep is the Top-k sweep without candidates (x = g + e written over E),
+// then one thread per message slot computes its coordinate, fetches x there and hands the pair to the server.
+#include "context.h"
+#include "scatter.cuh"
+
+namespace compams {
+
+__device__ __forceinline__ uint64_t philox4x64_10_first(uint64_t c0, uint64_t c1, uint64_t c2, uint64_t c3, uint64_t k0,
+                                                        uint64_t k1) {
+    const uint64_t M0 = 0xD2E7470EE14C6C93ull, M1 = 0xCA5A826395121157ull;
+    const uint64_t W0 = 0x9E3779B97F4A7C15ull, W1 = 0xBB67AE8584CAA73Bull;
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {
+            k0 += W0;
+            k1 += W1;
+        }
+        const uint64_t hi0 = __umul64hi(M0, c0), lo0 = M0 * c0;
+        const uint64_t hi1 = __umul64hi(M1, c2), lo1 = M1 * c2;
+        const uint64_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0;
+        c1 = lo1;
+        c2 = n2;
+        c3 = lo0;
+    }
+    return c0;
+}
+
+// Image of r under the permutation of {0, ..., m - 1} for (seed, step, worker, block); m < 2^32.
+__device__ __forceinline__ uint32_t randk_permute(uint32_t m, uint32_t r, uint64_t seed, uint64_t step, uint64_t worker,
+                                                  uint64_t block) {
+    int bits = 2;
+    while (bits < 32 && (1u << bits) < m) bits += 2;
+    const int w = bits >> 1;
+    const uint32_t mask = (1u << w) - 1u;
+    uint32_t x = r;
+    do {
+        uint32_t L = x >> w, R = x & mask;
+#pragma unroll 1
+        for (uint32_t round = 0; round < 4u; ++round) {
+            const uint32_t f = (uint32_t)philox4x64_10_first(R, round, block, worker, seed, step) & mask;
+            const uint32_t nR = L ^ f;
+            L = R;
+            R = nR;
+        }
+        x = (L << w) | R;
+    } while (x >= m);  // at most a few rounds on average: the domain is less than four times m
+    return x;
+}
+
+// One thread per message slot of this handle's t.n workers (worker il of the handle is worker row0 + il of the job).
+__global__ void __launch_bounds__(kThreads) randk_emit_kernel(Tables t, TopkBuffers b, int32_t row0, uint64_t seed,
+                                                              uint64_t step, int deliver) {
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool valid = p < (int64_t)t.n * b.K;
+    int32_t j = 0;
+    uint32_t xbits = 0;
+    int64_t il = 0;
+    if (valid) {
+        il = p / b.K;
+        const int64_t q = p % b.K;  // slot within the worker's row; its block by bisection of the slot offsets
+        int lo = 0, hi = t.M - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (__ldg(b.seg_off + mid) <= q) lo = mid; else hi = mid - 1;
+        }
+        const int64_t o = __ldg(t.off + lo);
+        const uint32_t len = (uint32_t)(__ldg(t.off + lo + 1) - o);
+        const uint32_t r = (uint32_t)(q - __ldg(b.seg_off + lo));
+        j = (int32_t)(o + randk_permute(len, r, seed, step, (uint64_t)(row0 + il), (uint64_t)lo));
+        xbits = __float_as_uint(b.E[(size_t)il * (size_t)t.d + (size_t)j]);  // the sweep left x = g + e there
+        const size_t slot = (size_t)(row0 + il) * (size_t)b.K + (size_t)q;
+        b.idx[slot] = j;
+        b.val[slot] = __uint_as_float(xbits);
+    }
+    if (deliver) scatter_warp(t, b, valid, j, xbits, il);
+}
+
+cudaError_t launch_randk_emit(compams_context* c, bool deliver) {
+    const int64_t count = (int64_t)c->n * c->K;
+    const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
+    randk_emit_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, c->row0, c->seed, c->iter, deliver ? 1 : 0);
+    return counted(c, cudaGetLastError());
+}
+
+}  // namespace compams

@@ -32,6 +32,7 @@
 #include <cooperative_groups.h>
 
 #include "context.h"
+#include "scatter.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 6) topk_sweep_kernel(Tables t, TopkB
 // select: exact Top-k inside the candidate list
 
 // Prediction for the next step's sweep, from this step's threshold key `tau` and the bin edge
-// `edge` at or above which about 2.5 k_b keys lay: the threshold keeps rising while the error
+// `edge` at or above which about the wanted number of candidates (want_candidates) lay: the threshold keeps rising while the error
 // accumulators fill, so tau_hat follows half of the last rise. `sel_shift` sizes the bins of the
 // next select so that the expected threshold lands near the middle of its 4096 bins.
 __device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_t edge, bool enabled) {
@@ -204,10 +205,35 @@ __device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_
     if (next >= 0x7f800000u) next = edge;
     const uint32_t tau_pred = tau + rise;
     uint32_t span = tau_pred > next ? tau_pred - next : 1u;
-    if (span < 2048u) span = 2048u;
+    // ... but never so fine that the bins end close above the prediction: they cover at least a quarter of a
+    // binade (values up to about 19 % above tau_hat), so a threshold that lands higher than predicted - gradients
+    // that alternate between two levels do that - is still found inside the list
+    if (span < (1u << 19)) span = 1u << 19;
     st->sel_shift = 32u - (uint32_t)__clz(span >> 11);  // smallest S with span >> S < 2048
     st->tau_hat = enabled ? next : kNoPrediction;
     st->tau_prev = tau;
+}
+
+// How many candidates the next step's predicted threshold should let through for a segment that keeps kb: the
+// count of keys above a fixed threshold moves by about sqrt(kb) from one step to the next (eight of those are
+// allowed for), plus a quarter of kb for drift of the gradient scale. A segment whose list came up short gets
+// its margin doubled (`boost` times, at most three); the doubling is taken back one step at a time after 32
+// selections in a row were decided inside the list. Long lists thus carry about 1.26 kb entries, short ones
+// (kb = 50: 170) proportionally more.
+__device__ __forceinline__ uint32_t want_candidates(uint32_t kb, uint32_t boost) {
+    const uint32_t margin = ((kb >> 2) + (uint32_t)(8.0f * sqrtf((float)kb)) + 32u) << (boost < 3u ? boost : 3u);
+    const uint32_t most = 4u * kb + 512u;  // half the list's capacity
+    return kb + (margin < most - kb ? margin : most - kb);
+}
+__device__ __forceinline__ void margin_came_up_short(SegState* st) {
+    if (st->boost < 3u) ++st->boost;
+    st->streak = 0u;
+}
+__device__ __forceinline__ void margin_held(SegState* st) {
+    if (++st->streak >= 32u) {
+        st->streak = 0u;
+        if (st->boost) --st->boost;
+    }
 }
 
 constexpr int kSelUnroll = 4;   // candidate loads in flight per thread while scanning a list
@@ -279,9 +305,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     __shared__ uint32_t scratch[kSelWarps];
     __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt;
     const int lane = threadIdx.x & 31;
-    const size_t item = blockIdx.x;
-    const int i = (int)(item / (size_t)nlist);
-    const int seg = seg_list[item % (size_t)nlist];
+    const int i = (int)(blockIdx.x / (unsigned)nlist);
+    const int seg = seg_list[blockIdx.x % (unsigned)nlist];
     const size_t sg = (size_t)i * t.nseg + seg;
     const SegInfo* si = t.segs + seg;
     SegState* st = b.seg + sg;
@@ -294,6 +319,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
             if (tau_hat != kNoPrediction) atomicAdd(b.status + (c < kb ? 3 : 4), 1u);  // too few / too many candidates
+            if (tau_hat != kNoPrediction && c < kb) margin_came_up_short(st);
         }
         return;
     }
@@ -327,7 +353,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     uint32_t total;
     {
         const BinScan sc = scan_from_top(local, kSelBins, scratch, &total);
-        const uint32_t want = 2u * kb + (kb >> 1);
+        const uint32_t want = want_candidates(kb, st->boost);
         if (threadIdx.x == 0) sh_edge[0] = 0xffffffffu;  // "fewer than `want` candidates"
         __syncthreads();
         locate(local, kSelBins, sc, kb, sh_bin);
@@ -451,11 +477,12 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
             const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
             edge = ew < 0x7f7fffffull ? (uint32_t)ew : 0x7f7fffffu;
         } else {
-            // fewer than 2.5 k_b candidates: reach further down next time, by half the distance to the threshold
+            // fewer candidates than wanted: reach further down next time, by half the distance to the threshold
             const uint32_t gap = ((tau - tau_hat) >> 1) + (1u << 16);
             edge = tau_hat > gap ? tau_hat - gap : 0u;
         }
         predict_next(st, tau, edge, true);
+        margin_held(st);
         st->fallback = 0u;
         atomicAdd(b.status + 2, 1u);  // selections decided inside their candidate list
     }
@@ -497,6 +524,7 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
             st->fallback = 1u;
             atomicAdd(b.dense_count, 1u);
             if (tau_hat != kNoPrediction) atomicAdd(b.status + (c < kb ? 3 : 4), 1u);  // too few / too many candidates
+            if (tau_hat != kNoPrediction && c < kb) margin_came_up_short(st);
         }
         return;
     }
@@ -544,7 +572,7 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
     __syncthreads();
     uint32_t total;
     const BinScan sc = scan_from_top<kThreads>(local, kSelBins, scratch, &total);
-    const uint32_t want = 2u * kb + (kb >> 1);
+    const uint32_t want = want_candidates(kb, st->boost);
     if (threadIdx.x == 0) sh_edge[0] = 0xffffffffu;  // "fewer than `want` candidates"
     __syncthreads();
     locate<kThreads>(local, kSelBins, sc, kb, sh_bin);
@@ -601,45 +629,45 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
     uint2* gsurv = b.sel_surv + item * kSurvCapBig;
     uint32_t* gscnt = b.sel_ticket + 2 * item + 1;  // survivors appended so far (second word of the pair)
 
-    // first pass over the slice (from L2): how many winners, so that they get one contiguous slot range
-    uint32_t mine = 0;
-    for (uint32_t p = lo + threadIdx.x; p < hi; p += kThreads) {
-        const uint32_t dg = offset_digit(list[p].y, tau_hat, S);
-        mine += (dg > b0 || (take_all0 && dg == b0)) ? 1u : 0u;
-    }
-    uint32_t my_winners;
-    block_inclusive_scan(mine, scratch, &my_winners);
-    if (threadIdx.x == 0) {
-        sh_base = my_winners ? atomicAdd(&st->emit_count, my_winners) : 0u;
-        sh_wcnt = 0u;
-    }
-    __syncthreads();
-    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {
+    // one pass over the slice, a chunk of kSelUnroll candidates per thread at a time: the chunk's winners are
+    // counted (a scan over the CTA), get one contiguous range of message slots with a single atomic, and are
+    // written there
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kThreads) {  // uniform trip count: the loop holds barriers
         uint2 cvs[kSelUnroll];
 #pragma unroll
         for (int u = 0; u < kSelUnroll; ++u) {
             const uint32_t p = p0 + u * kThreads + threadIdx.x;
             cvs[u] = p < hi ? list[p] : make_uint2(0u, 0xffffffffu);
         }
+        uint32_t winmask = 0, keepmask = 0;
 #pragma unroll
         for (int u = 0; u < kSelUnroll; ++u) {
-            const uint2 cv = cvs[u];
-            const bool valid = cv.y != 0xffffffffu;
-            const uint32_t dg = valid ? offset_digit(cv.y, tau_hat, S) : 0u;
-            const bool win = valid && (dg > b0 || (take_all0 && dg == b0));
-            const bool keep = valid && !take_all0 && dg == b0;
-            const uint32_t wpos = sh_base + warp_slot(win, &sh_wcnt, lane);
-            if (win) {
+            const bool valid = cvs[u].y != 0xffffffffu;
+            const uint32_t dg = valid ? offset_digit(cvs[u].y, tau_hat, S) : 0u;
+            if (valid && (dg > b0 || (take_all0 && dg == b0))) winmask |= 1u << u;
+            if (valid && !take_all0 && dg == b0) keepmask |= 1u << u;
+        }
+        const uint32_t mine = (uint32_t)__popc(winmask);
+        uint32_t chunk_winners;
+        const uint32_t incl = block_inclusive_scan(mine, scratch, &chunk_winners);
+        if (threadIdx.x == 0) sh_base = chunk_winners ? atomicAdd(&st->emit_count, chunk_winners) : 0u;
+        __syncthreads();
+        uint32_t wpos = sh_base + incl - mine;
+#pragma unroll
+        for (int u = 0; u < kSelUnroll; ++u) {
+            if ((winmask >> u) & 1u) {
                 if (wpos < kb) {
-                    b.idx[slot0 + wpos] = (int32_t)cv.x;
-                    b.val[slot0 + wpos] = __uint_as_float(cv.y);
+                    b.idx[slot0 + wpos] = (int32_t)cvs[u].x;
+                    b.val[slot0 + wpos] = __uint_as_float(cvs[u].y);
                 } else {
                     atomicOr(b.status, 1u);
                 }
+                ++wpos;
             }
+            const bool keep = (keepmask >> u) & 1u;
             if (__any_sync(0xffffffffu, keep)) {  // rare: only the threshold bin's candidates
                 const uint32_t spos = warp_slot(keep, gscnt, lane);
-                if (keep && spos < (uint32_t)kSurvCapBig) gsurv[spos] = cv;
+                if (keep && spos < (uint32_t)kSurvCapBig) gsurv[spos] = cvs[u];
             }
         }
     }
@@ -777,11 +805,12 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
             const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
             edge = ew < 0x7f7fffffull ? (uint32_t)ew : 0x7f7fffffu;
         } else {
-            // fewer than 2.5 k_b candidates: reach further down next time, by half the distance to the threshold
+            // fewer candidates than wanted: reach further down next time, by half the distance to the threshold
             const uint32_t gap = ((tau - tau_hat) >> 1) + (1u << 16);
             edge = tau_hat > gap ? tau_hat - gap : 0u;
         }
         predict_next(st, tau, edge, true);
+        margin_held(st);
         st->fallback = 0u;
         atomicAdd(b.status + 2, 1u);  // selections decided inside their candidate list
     }
@@ -877,9 +906,9 @@ __device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b
         }
     }
     if (PASS == 1) {
-        // the highest pass-1 bin edge at or above which at least 2.5 k_b keys lie (0 if there are fewer);
-        // a candidate path that gave up may have handed out message slots: start over
-        const uint32_t want = 2u * kb + (kb >> 1);
+        // the highest pass-1 bin edge at or above which at least the wanted number of candidates lie (0 if there
+        // are fewer); a candidate path that gave up may have handed out message slots: start over
+        const uint32_t want = want_candidates(kb, st->boost);
         if (threadIdx.x == 0) {
             st->emit_count = 0u;
             if (total < want) st->edge = 0u;
@@ -1027,6 +1056,20 @@ __device__ __forceinline__ void dense_ties(const Tables& t, const TopkBuffers& b
     if (threadIdx.x == 0 && taken < want) atomicOr(b.status, 1u);
 }
 
+// Closes the step for one large-block segment: exactly k_b entries must have been emitted; the counters go
+// back to their resting values.
+__device__ __forceinline__ void close_segment(const TopkBuffers& b, const SegInfo* si, SegState* st) {
+    const bool dense = st->fallback != 0u;
+    const uint32_t ties = (dense && st->need_order) ? st->ties_take : 0u;
+    if (st->emit_count + ties != si->kb) atomicOr(b.status, 1u);
+    if (dense) atomicAdd(b.status + 1, 1u);              // selections decided by the dense passes
+    if (dense && si->cap) atomicSub(b.dense_count, 1u);  // back to the number of blocks that never predict
+    st->emit_count = 0u;
+    st->cand_count = 0u;
+    st->fallback = si->cap ? 0u : 1u;  // blocks without a candidate buffer always take the dense passes
+    st->need_order = 0u;
+}
+
 // All dense passes in one cooperative launch: the grid is resident as a whole and the passes are
 // separated by grid-wide barriers. When no segment is marked every CTA returns at once, so in the
 // steady state the dense path costs one empty launch per step.
@@ -1161,59 +1204,26 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 }
 
 // ------------------------------------------------------------------------------------------
-// scatter: acc[j] += x_ij over all kept (i, j); binary64 atomics, exact hence order-independent.
-// The same walk zeroes e at the kept coordinates (they were left holding x by the sweep).
+// scatter: the kept (index, value) pairs of the messages are handed to the server grouped by coordinate
+// range, and the kept coordinates recorded for the residual update.
 
-__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count, int32_t row0) {
+// All messages at once (`count` pairs of every worker the server averages over; E and the kept map hold
+// the t.n workers of this handle, whose first is worker row0). The first n * nseg threads also close the
+// step for one large-block segment each.
+__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count, int32_t row0,
+                                                                int close) {
     dependency_wait();
     allow_dependents();
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    // the first n * nseg threads also close the step for one large-block segment each: exactly k_b
-    // entries must have been emitted; counters go back to their resting values
-    if (p < (int64_t)t.n * t.nseg) {
-        const SegInfo* si = t.segs + (p % t.nseg);
-        SegState* st = b.seg + p;
-        const bool dense = st->fallback != 0u;
-        const uint32_t ties = (dense && st->need_order) ? st->ties_take : 0u;
-        if (st->emit_count + ties != si->kb) atomicOr(b.status, 1u);
-        if (dense) atomicAdd(b.status + 1, 1u);              // selections decided by the dense passes
-        if (dense && si->cap) atomicSub(b.dense_count, 1u);  // back to the number of blocks that never predict
-        st->emit_count = 0u;
-        st->cand_count = 0u;
-        st->fallback = si->cap ? 0u : 1u;  // blocks without a candidate buffer always take the dense passes
-        st->need_order = 0u;
-    }
-    // one (index, value) pair per thread. The pair joins the bucket of its coordinate range (slots
-    // handed out with one atomic per warp and bucket); e is zeroed at the kept coordinate.
+    if (close && p < (int64_t)t.n * t.nseg) close_segment(b, t.segs + (p % t.nseg), b.seg + p);
     const bool valid = p < count;
     int32_t j = 0;
-    uint32_t xbits = 0, T = 0xffffffffu;
+    uint32_t xbits = 0;
     if (valid) {
         j = __ldg(b.idx + p);
         xbits = __float_as_uint(__ldg(b.val + p));
-        T = (uint32_t)j / (uint32_t)kBucketSpan;
     }
-    const int lane = threadIdx.x & 31;
-    const unsigned peers = __match_any_sync(0xffffffffu, T);
-    uint32_t base = 0;
-    const int leader = __ffs(peers) - 1;
-    if (valid && lane == leader) base = atomicAdd(b.bcount + T, (uint32_t)__popc(peers));
-    base = __shfl_sync(0xffffffffu, base, leader);
-    if (!valid) return;
-    const uint32_t pos = base + (uint32_t)__popc(peers & ((1u << lane) - 1u));
-    if (pos < (uint32_t)b.bucket_cap) {
-        b.bucket[(size_t)T * (size_t)b.bucket_cap + pos] = make_uint2((uint32_t)j % (uint32_t)kBucketSpan, xbits);
-    } else {  // a coordinate range kept by far more entries than average: binary64 atomics instead
-        atomicAdd(b.acc + j, (double)__uint_as_float(xbits));
-        b.bdirty[T] = 1u;
-    }
-    // the coordinate's e becomes 0 (the residual update: e = x - x): recorded in the kept map, applied when E is next read
-    // (`count` covers the messages of every worker the server averages over; E and the kept map hold
-    // the t.n workers of this handle, whose first is worker row0)
-    const int64_t il = p / b.K - row0;
-    if (il < 0 || il >= t.n) return;
-    const int64_t f = il * t.d + j;  // the element's index in E, [n, d] flattened
-    atomicOr(b.kept_cur + (size_t)(f >> 5), 1u << (uint32_t)(f & 31));
+    scatter_warp(t, b, valid, j, xbits, valid ? p / b.K - row0 : -1);
 }
 
 // E holds x at the coordinates kept in the last step: zero them (Algorithm 2, the residual update), one thread per word.
@@ -1314,14 +1324,15 @@ cudaError_t launch_topk_materialize(compams_context* c) {
     return counted(c, cudaGetLastError());
 }
 
-cudaError_t launch_topk_scatter(compams_context* c) {
+cudaError_t launch_topk_scatter(compams_context* c, bool close) {
     // one thread per message entry of every worker (>= n * nseg: every block keeps at least one entry)
     const int64_t count = (int64_t)c->n_total * c->K;
     const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
     // (a sharded handle's exchange sits in front of this kernel: a plain launch waits for it)
     if (c->chain && c->n == c->n_total)
-        return counted(c, launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count, c->row0));
-    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, c->row0);
+        return counted(c, launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count, c->row0,
+                                       close ? 1 : 0));
+    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, c->row0, close ? 1 : 0);
     return counted(c, cudaGetLastError());
 }
 

@@ -6,8 +6,9 @@ gradients and error accumulators never leave its GPU. One step is compress() on 
 all-gather of the message buffers - (index, value) pairs for Top-k, sign words and scales for
 Block-Sign: n_total * K * 8 bytes or n_total * (d / 8 + 4 M) bytes in total - and apply() on every
 rank. Every rank plays the server on its own replica of theta, m, v, v-hat; the update is a
-deterministic function of the gathered messages, so the replicas stay bit-identical and theta is
-never broadcast. The collective is torch.distributed's (NCCL between GPUs); the gathered rows land in
+function of the gathered messages alone (the sum over workers is exact, hence order-free, while the
+magnitudes met at one coordinate lie within about 2^24 of one another), so the replicas stay bit-identical
+and theta is never broadcast. The collective is torch.distributed's (NCCL between GPUs); the gathered rows land in
 this rank's own memory and the kernels read them with ordinary loads.
 """
 from __future__ import annotations
@@ -39,9 +40,19 @@ def exchange(buffers: Sequence[torch.Tensor], first_row: int, rows: int, group=N
     world = dist.get_world_size(group)
     if world == 1:
         return
+    on_device = dist.get_backend(group) == "nccl"
     for buf in buffers:
         if buf.shape[0] != world * rows:
             raise ValueError("a buffer of %d rows cannot hold %d rows from each of %d ranks" % (buf.shape[0], rows, world))
+        if buf.is_cuda and not on_device:
+            # a group whose backend moves host memory only (gloo): this rank's rows go to the host (the copy waits
+            # for the work that wrote them, on the current stream), the gathered rows come back from a pinned buffer
+            mine = buf[first_row:first_row + rows].cpu()
+            whole = torch.empty(buf.shape, dtype=buf.dtype, pin_memory=True)
+            dist.all_gather_into_tensor(whole.view(-1), mine.view(-1), group=group)
+            buf.copy_(whole, non_blocking=True)
+            torch.cuda.current_stream().synchronize()  # `whole` is released on return
+            continue
         mine = buf[first_row:first_row + rows].clone()  # the messages are small next to the gradients
         dist.all_gather_into_tensor(buf.view(-1), mine.view(-1), group=group)
 
@@ -72,6 +83,11 @@ class ShardedCompAMS:
     def message_bytes_per_step(self) -> int:
         """Bytes this rank receives from the others in one step's exchange."""
         return sum(b[0].numel() * b.element_size() for b in self.opt.message_buffers()) * (self.opt.n_total - self.opt.n)
+
+    def total_message_bytes_per_step(self) -> int:
+        """Bytes of all workers' compressed gradients of one step: n_total K 8 for Top-k and Random-k (a 32-bit
+        index and a 32-bit value per kept coordinate), n_total (4 W + 4 M) for Block-Sign (W sign words, M scales)."""
+        return sum(b[0].numel() * b.element_size() for b in self.opt.message_buffers()) * self.opt.n_total
 
     def close(self) -> None:
         self.opt.close()

@@ -22,6 +22,7 @@ import torch
 
 TOPK = 0
 BLOCKSIGN = 1
+RANDK = 2
 
 Shape = Tuple[int, ...]
 

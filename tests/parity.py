@@ -10,7 +10,7 @@ import numpy as np
 import torch
 
 import oracle
-from paper_2205_05632_b200 import BLOCKSIGN, TOPK, CompAMS
+from paper_2205_05632_b200 import BLOCKSIGN, RANDK, TOPK, CompAMS
 
 ATOL, RTOL = 1e-7, 1e-6
 
@@ -58,7 +58,8 @@ def unpack_sign_bits(bits: np.ndarray, word_off: np.ndarray, block_offsets: np.n
 class Pair:
     """A CUDA optimizer and an oracle built from the same arguments."""
 
-    def __init__(self, n, d, block_offsets, compressor, k_ratio=1.0, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8):
+    def __init__(self, n, d, block_offsets, compressor, k_ratio=1.0, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
+                 seed=None):
         self.n, self.d = n, d
         self.offsets = np.asarray(block_offsets, dtype=np.int64)
         self.compressor = compressor
@@ -66,7 +67,10 @@ class Pair:
         self.gpu = CompAMS(n, d, self.offsets, compressor, k_ratio, **hp)
         self.cpu = oracle.Oracle(n, d, self.offsets, compressor, k_ratio, **hp)
         sizes = np.diff(self.offsets)
-        self.identity = compressor == TOPK and all(oracle.kept_per_block(k_ratio, int(s)) == int(s) for s in sizes)
+        if seed is not None:  # Random-k: the same seed for the index sets on both sides
+            self.gpu.set_seed(seed)
+            self.cpu.set_seed(seed)
+        self.identity = compressor in (TOPK, RANDK) and all(oracle.kept_per_block(k_ratio, int(s)) == int(s) for s in sizes)
         self.step_no = 0
         self.inexact = {}
 
@@ -84,7 +88,7 @@ class Pair:
         self.cpu.step(np.ascontiguousarray(G.detach().float().cpu().numpy()), self.theta_cpu)
         assert self.gpu.check_status() == 0
         cnt = self.inexact
-        if self.compressor == TOPK and not self.identity:
+        if self.compressor in (TOPK, RANDK) and not self.identity:
             idx = self.gpu.buffer("topk_idx").cpu().numpy()
             val = self.gpu.buffer("topk_val")
             order = np.argsort(idx, axis=1, kind="stable")

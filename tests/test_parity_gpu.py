@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2205_05632_b200 import BLOCKSIGN, TOPK, CompAMS, CompAMSError
+from paper_2205_05632_b200 import BLOCKSIGN, RANDK, TOPK, CompAMS, CompAMSError
 from paper_2205_05632_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -12,6 +12,8 @@ pytestmark = pytest.mark.gpu
 def _pair_run(n, d, offsets, comp, ratio, make_g, steps=4, theta_sigma=0.1, check_e_every=1, **hp):
     from parity import Pair
     gen = torch.Generator(device="cuda").manual_seed(1234)
+    if comp == RANDK:
+        hp.setdefault("seed", 2022)
     p = Pair(n, d, offsets, comp, ratio, **hp)
     try:
         p.start(theta_sigma * torch.randn(d, generator=gen, device="cuda"))
@@ -321,6 +323,27 @@ def test_topk_candidate_path_is_taken_in_steady_state():
         p.close()
 
 
+@pytest.mark.parametrize("d", [40 * 8192 + 321, (1 << 21) + 5])
+def test_topk_candidate_path_survives_gradients_that_alternate_between_two_batches(d):
+    # the same two gradient tensors in turn (what a benchmark ring does, and what a data loader with two
+    # shards does): the threshold then alternates between two levels instead of drifting. The prediction must
+    # keep the selection inside the candidate lists (short list: one CTA; long list: slices) - and stay exact
+    from parity import Pair
+    n = 4
+    gen = torch.Generator(device="cuda").manual_seed(8)
+    ring = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(2)]
+    p = Pair(n, d, [0, d], TOPK, 0.01)
+    try:
+        p.start(torch.zeros(d, device="cuda"))
+        for t in range(12):
+            p.step(ring[t % 2], check_e=(t % 4 == 3))
+        st = _status(p.gpu)
+        assert st[0] == 0 and st[1] + st[2] == 12 * n
+        assert st[1] <= 3 * n, "dense passes ran on %d of %d selections: %r" % (st[1], 12 * n, st)
+    finally:
+        p.close()
+
+
 def test_topk_prediction_failures_fall_back_exactly():
     # the gradient scale jumps by orders of magnitude between steps: too few candidates, too many,
     # thresholds far above the predicted range - every case must still give the exact Top-k
@@ -440,6 +463,57 @@ def test_calls_out_of_order_are_rejected():
         assert torch.equal(theta, theta_ref) and torch.equal(opt.buffer("E"), ref.buffer("E"))
         opt.close()
         ref.close()
+
+
+# ------------------------------------------------------------------ Random-k
+
+@pytest.mark.parametrize("n", [1, 3])
+@pytest.mark.parametrize("ratio", [0.01, 0.3, 1.0])
+def test_randk_ragged_blocks(n, ratio):
+    d = RAGGED[-1]
+    _pair_run(n, d, RAGGED, RANDK, ratio, _randn(n, d), steps=5)
+
+
+@pytest.mark.parametrize("d", [1, 2, 5, 33, 4097, 8193, 3 * 8192 + 2])
+def test_randk_single_block_sizes(d):
+    _pair_run(2, d, [0, d], RANDK, 0.1, _randn(2, d), steps=3)
+
+
+def test_randk_resnet18_shapes_layerwise_and_whole_vector():
+    # large enough that the step is overlapped (groups of workers, messages delivered behind the sweeps)
+    w = W.config2("cuda")
+    theta = w.start()
+    from parity import Pair
+    for offs, ratio in ((w.block_offsets, 0.01), (np.array([0, w.d]), 0.001)):
+        p = Pair(8, w.d, offs, RANDK, ratio, seed=5)
+        try:
+            p.start(theta)
+            for t in range(4):
+                p.step(w.grads()[:8].contiguous(), check_e=(t % 2 == 1))
+        finally:
+            p.close()
+
+
+def test_randk_sets_follow_seed_and_iteration_count():
+    n, d = 2, 50000
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    G = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(3)]
+
+    def run(seed, start):
+        opt = CompAMS(n, d, [0, 20000, d], RANDK, 0.01)
+        opt.set_seed(seed, start)
+        theta = torch.zeros(d, device="cuda")
+        sets = []
+        for g in G:
+            opt.step(g, theta)
+            sets.append(torch.sort(opt.buffer("topk_idx"), dim=1).values.clone())
+        opt.close()
+        return sets
+
+    a, b, c, late = run(1, 0), run(1, 0), run(2, 0), run(1, 1)
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+    assert not torch.equal(a[0], c[0])
+    assert torch.equal(a[1], late[0]) and torch.equal(a[2], late[1])  # iteration t + 1 of one run = iteration t of a run started one later
 
 
 # ------------------------------------------------------------------ checkpoint / restore, traffic accounting
