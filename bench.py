@@ -411,7 +411,7 @@ def main():
         # ---- per-kernel breakdown of the step, from a few extra steps with an event pair around every launch
         opt.set_profiling(KERNELS["topk"])
         for t in range(3):
-            opt.step(ring[t % 2], theta)
+            opt.step(ring[(args.warmup + args.steps + t) % 2], theta)  # the ring goes on in step
         per_kernel = {}
         for k in KERNELS["topk"]:
             ms, cnt = opt.kernel_time(k)

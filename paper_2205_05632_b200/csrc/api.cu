@@ -258,9 +258,10 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &t.tile_ties, c->randk ? 1 : (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &t.cand, (size_t)n * (size_t)t.cand_total, false));
         RC(dev_alloc(c, &t.acc, (size_t)d));
-        t.map_words = ((int64_t)n * d + 31) / 32;
-        RC(dev_alloc(c, &c->keptmap[0], (size_t)t.map_words));
-        RC(dev_alloc(c, &c->keptmap[1], (size_t)t.map_words));
+        {
+            std::vector<uint32_t> none((size_t)n * (size_t)std::max(c->tab.nseg, 1), 0xffffffffu);
+            RC(dev_upload(c, &t.thr, none));
+        }
         {
             // kept entries are handed to the server grouped by coordinate range: room for four times the
             // average load of a bucket, the rare excess goes through the binary64 accumulator
@@ -355,20 +356,15 @@ int compress_device(compams_context* c, const void* grads) {
         RC(run_kernel(c, COMPAMS_K_BS_SCALES, [&] { return launch_bs_scales(c); }));
         return COMPAMS_OK;
     }
-    // kept coordinates are recorded in a bit map; their e is zeroed when E is next read (by the next
-    // sweep, or by topk_materialize when the caller asks for E)
-    c->map_cur ^= 1;
-    c->tk.kept_cur = c->keptmap[c->map_cur];
-    c->tk.kept_prev = c->e_mask_pending ? c->keptmap[c->map_cur ^ 1] : nullptr;
-    CU(cudaMemsetAsync(c->tk.kept_cur, 0, (size_t)c->tk.map_words * sizeof(uint32_t), c->stream));
+    // a selection leaves x in E at the coordinates it keeps, and the pair that delimits them; their e is zeroed
+    // when E is next read (by the next sweep, or by topk_materialize when the caller asks for E)
+    c->tk.use_thr = c->e_mask_pending ? 1 : 0;
     if (c->randk) {
-        // no selection: the sweep leaves x in E, then every message slot fetches the x of its drawn coordinate;
-        // with all workers in this handle the pairs go to the server in the same kernel, otherwise
+        // no selection: the sweep leaves x in E, then every message slot fetches the x of its drawn coordinate and
+        // zeroes it; with all workers in this handle the pairs go to the server in the same kernel, otherwise
         // compams_apply delivers the exchanged messages
-        const bool deliver = c->n == c->n_total;
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
-        RC(run_kernel(c, COMPAMS_K_RANDK_EMIT, [&] { return launch_randk_emit(c, deliver); }));
-        if (deliver) c->e_mask_pending = true;
+        RC(run_kernel(c, COMPAMS_K_RANDK_EMIT, [&] { return launch_randk_emit(c, c->n == c->n_total); }));
         return COMPAMS_OK;
     }
     if (c->tk.nsmall > 0) RC(run_kernel(c, COMPAMS_K_TOPK_SMALL, [&] { return launch_topk_small(c, grads); }));
@@ -376,6 +372,7 @@ int compress_device(compams_context* c, const void* grads) {
         RC(run_kernel(c, COMPAMS_K_TOPK_SWEEP, [&] { return launch_topk_sweep(c, grads); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_SELECT, [&] { return launch_topk_select(c); }));
         RC(run_kernel(c, COMPAMS_K_TOPK_DENSE, [&] { return launch_topk_dense(c); }));
+        c->e_mask_pending = true;
     }
     return COMPAMS_OK;
 }
@@ -386,10 +383,8 @@ int apply_device(compams_context* c, float* theta) {
         return run_kernel(c, COMPAMS_K_BS_APPLY, [&] { return launch_bs_apply(c, theta); });
     }
     // (a Random-k step with every worker in this handle has delivered its messages already)
-    if (!(c->randk && c->n == c->n_total)) {
+    if (!(c->randk && c->n == c->n_total))
         RC(run_kernel(c, COMPAMS_K_TOPK_SCATTER, [&] { return launch_topk_scatter(c, !c->randk); }));
-        c->e_mask_pending = true;
-    }
     RC(run_kernel(c, COMPAMS_K_AMSGRAD, [&] { return launch_amsgrad(c, theta); }));
     return COMPAMS_OK;
 }

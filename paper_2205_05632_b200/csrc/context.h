@@ -96,10 +96,9 @@ struct TopkBuffers {
     uint32_t* sel_ticket;      // [n * long lists, 2] slices arrived; threshold-bin candidates appended
     uint2* sel_surv;           // [n * long lists, kSurvCapBig] threshold-bin candidates of a long list
     double* acc;               // [d] binary64 accumulator, used only by entries that overflow their bucket
-    const uint32_t* kept_prev; // [map_words] bit i d + j: worker i kept coordinate j last step and its e is still
-                               // to be zeroed (null when E is up to date)
-    uint32_t* kept_cur;        // [map_words] receives this step's kept coordinates
-    int64_t map_words;         // 32-bit words of a kept map: ceil(n d / 32), one bit per element of E
+    uint32_t* thr;             // [n * nseg] bits of the magnitude from which on the segment's last selection kept
+                               // everything: E still holds x at those elements; their e is 0
+    int use_thr;               // 1: E holds the last step's x at the kept coordinates (the sweep treats them as 0)
     uint2* bucket;             // [nbucket, bucket_cap] (coordinate inside the bucket, bits of x) per kept entry
     uint32_t* bcount;          // [nbucket] entries appended this step (may exceed bucket_cap)
     uint32_t* bdirty;          // [nbucket] 1: some entries of this bucket went to acc instead
@@ -148,8 +147,6 @@ struct compams_context {
     std::vector<compams::SegState> seg_init_host;  // Top-k: the segments' state before the first step (set_state restores it)
     uint32_t dense_count_init = 0;
     uint64_t steps_done = 0;
-    uint32_t* keptmap[2] = {nullptr, nullptr};  // Top-k: kept maps of this and the previous step
-    int map_cur = 0;
     bool e_mask_pending = false;  // Top-k: E still holds x at the coordinates kept in the last step
     int dense_grid = 0;  // CTAs of the cooperative dense-pass kernel (0: not yet sized)
     float* scales[2] = {nullptr, nullptr};

@@ -8,7 +8,8 @@
 // word of Philox4x64-10 (Salmon, Moraes, Dror, Shaw, SC 2011) at counter (right half, round, b, i) under
 // key (seed, t). Being the image of k_b distinct inputs under a bijection, the set has exactly k_b members
 // and needs no selection pass: the sweep is the Top-k sweep without candidates (x = g + e written over E),
-// then one thread per message slot computes its coordinate, fetches x there and hands the pair to the server.
+// then one thread per message slot computes its coordinate, fetches x there, zeroes it (the residual of a kept
+// coordinate) and hands the pair to the server.
 #include "context.h"
 #include "scatter.cuh"
 
@@ -77,12 +78,14 @@ __global__ void __launch_bounds__(kThreads) randk_emit_kernel(Tables t, TopkBuff
         const uint32_t len = (uint32_t)(__ldg(t.off + lo + 1) - o);
         const uint32_t r = (uint32_t)(q - __ldg(b.seg_off + lo));
         j = (int32_t)(o + randk_permute(len, r, seed, step, (uint64_t)(row0 + il), (uint64_t)lo));
-        xbits = __float_as_uint(b.E[(size_t)il * (size_t)t.d + (size_t)j]);  // the sweep left x = g + e there
+        float* ex = b.E + (size_t)il * (size_t)t.d + (size_t)j;
+        xbits = __float_as_uint(*ex);  // the sweep left x = g + e there
+        *ex = 0.0f;                    // the residual update at a kept coordinate: e = x - x
         const size_t slot = (size_t)(row0 + il) * (size_t)b.K + (size_t)q;
         b.idx[slot] = j;
         b.val[slot] = __uint_as_float(xbits);
     }
-    if (deliver) scatter_warp(t, b, valid, j, xbits, il);
+    if (deliver) scatter_warp(b, valid, j, xbits);
 }
 
 cudaError_t launch_randk_emit(compams_context* c, bool deliver) {

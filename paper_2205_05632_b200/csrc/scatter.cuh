@@ -5,28 +5,20 @@
 
 namespace compams {
 
-// A kept (coordinate, value) pair of worker `il` (its index among this handle's workers; pairs of other
-// shards' workers pass a value outside [0, n)) reaches the server: it joins the bucket of its coordinate
-// range at position `pos` - or, when the bucket is full, the binary64 accumulator - and, for this handle's
-// own workers, the coordinate's e becomes 0 (the residual update: e = x - x), recorded in the kept map and
-// applied when E is next read.
-__device__ __forceinline__ void deliver_pair(const Tables& t, const TopkBuffers& b, uint32_t T, uint32_t pos, int32_t j,
-                                             uint32_t xbits, int64_t il) {
+// A kept (coordinate, value) pair reaches the server: it joins the bucket of its coordinate range at position
+// `pos` or, when the bucket is full, the binary64 accumulator.
+__device__ __forceinline__ void deliver_pair(const TopkBuffers& b, uint32_t T, uint32_t pos, int32_t j, uint32_t xbits) {
     if (pos < (uint32_t)b.bucket_cap) {
         b.bucket[(size_t)T * (size_t)b.bucket_cap + pos] = make_uint2((uint32_t)j % (uint32_t)kBucketSpan, xbits);
     } else {  // a coordinate range kept by far more entries than average: binary64 atomics instead
         atomicAdd(b.acc + j, (double)__uint_as_float(xbits));
         b.bdirty[T] = 1u;
     }
-    if (il < 0 || il >= t.n) return;
-    const int64_t f = il * t.d + j;  // the element's index in E, [n, d] flattened
-    atomicOr(b.kept_cur + (size_t)(f >> 5), 1u << (uint32_t)(f & 31));
 }
 
 // One pair per thread, the whole warp together: the lanes whose pairs fall into the same bucket get their
 // slots with one atomic.
-__device__ __forceinline__ void scatter_warp(const Tables& t, const TopkBuffers& b, bool valid, int32_t j, uint32_t xbits,
-                                             int64_t il) {
+__device__ __forceinline__ void scatter_warp(const TopkBuffers& b, bool valid, int32_t j, uint32_t xbits) {
     const uint32_t T = valid ? (uint32_t)j / (uint32_t)kBucketSpan : 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const unsigned peers = __match_any_sync(0xffffffffu, T);
@@ -35,7 +27,7 @@ __device__ __forceinline__ void scatter_warp(const Tables& t, const TopkBuffers&
     if (valid && lane == leader) base = atomicAdd(b.bcount + T, (uint32_t)__popc(peers));
     base = __shfl_sync(0xffffffffu, base, leader);
     if (!valid) return;
-    deliver_pair(t, b, T, base + (uint32_t)__popc(peers & ((1u << lane) - 1u)), j, xbits, il);
+    deliver_pair(b, T, base + (uint32_t)__popc(peers & ((1u << lane) - 1u)), j, xbits);
 }
 
 }  // namespace compams

@@ -27,8 +27,12 @@
 //     ties          takes the lowest-index threshold ties, tile by tile in index order
 //   topk_scatter    closes the step per segment (count check, counters reset) and walks the
 //                   (index, value) messages: each pair is appended to the bucket of its coordinate range
-//                   for the server kernel (the server's average) and marked in the kept map: its e is 0 (the residual update:
-//                   e = x - x), applied when E is next read (next sweep, or topk_materialize)
+//                   for the server kernel (the server's average)
+//   The residual update at a kept coordinate (e = x - x = 0) is deferred: E keeps x there, and every selection
+//   leaves one magnitude per segment such that the kept elements are exactly those with |x| at or above it;
+//   whoever reads E next - the next sweep, or topk_materialize - treats them as 0. Where a selection cuts through
+//   a group of equal magnitudes (some kept, some not), it zeroes the few kept ones in E itself and leaves the
+//   next larger magnitude.
 #include <cooperative_groups.h>
 
 #include "context.h"
@@ -74,23 +78,20 @@ __device__ __forceinline__ void load_x_tile(const float* __restrict__ e, int len
 // ------------------------------------------------------------------------------------------
 // sweep: x = g + e -> E; keys >= tau_hat go to the candidate list
 
+// "Nothing kept": as a float this pattern is a NaN, which no magnitude reaches.
+constexpr uint32_t kNothingKept = 0xffffffffu;
+
 // One tile of the sweep. The tile starts at r0 (relative to the block), which is the block's tile
 // boundary shifted down to a 128-byte line of G and E: r0 may be negative and the tile may reach
-// past the block; such coordinates are skipped. `row0` is the index of the block's first element
-// in E ([n, d] flattened), which is also its bit in the kept map; row0 + r0 is a multiple of 32.
+// past the block; such coordinates are skipped.
+// `kept_from`: elements of E whose magnitude is at or above it were kept by the last step's selection and still
+// hold x; their e is 0 (one float comparison: the key order is the order of |x|).
 template <bool FULL, typename GT>
 __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float* __restrict__ e, int len, int r0,
-                                                int warp, int lane, uint32_t tau_hat, uint32_t coord0, int64_t row0,
+                                                int warp, int lane, uint32_t tau_hat, uint32_t coord0,
                                                 uint2* sh_cand, uint32_t* sh_cnt, uint32_t* g_cnt, uint2* g_out,
-                                                uint32_t cap, const uint32_t* __restrict__ kept, int64_t map_words) {
+                                                uint32_t cap, float kept_from) {
     const int cg_ = align_class(g + r0), ce = align_class(e + r0);
-    // kept map of this warp's 1024 elements: lane l fetches word l once and the iterations pick
-    // their nibbles with shuffles
-    uint32_t mapw = 0u;
-    if (kept != nullptr) {
-        const int64_t w = ((row0 + lane_r(r0, warp, 0, 0)) >> 5) + lane;
-        mapw = w < map_words ? __ldg(kept + w) : 0u;
-    }
     constexpr int NB = 2;  // iterations whose loads are in flight together
 #pragma unroll
     for (int bt = 0; bt < kIters / NB; ++bt) {
@@ -116,14 +117,12 @@ __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float*
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
             const int r = lane_r(r0, warp, bt * NB + u, lane);
-            // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, the residual update).
-            // Placed after the batch's loads have been issued: the shuffle waits for the map word.
-            const uint32_t kb4 =
-                (__shfl_sync(0xffffffffu, mapw, (bt * NB + u) * 4 + (lane >> 3)) >> ((lane & 7) * 4)) & 0xfu;
             float xs[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float ek = ((kb4 >> k) & 1u) ? 0.0f : lane_elem(ev[u], k);
+                // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, the residual update)
+                const float eo = lane_elem(ev[u], k);
+                const float ek = fabsf(eo) >= kept_from ? 0.0f : eo;
                 xs[k] = __fadd_rn(lane_elem(gv[u], k), ek);  // the corrected-gradient step: x = g + e
                 if ((FULL || (unsigned)(r + k) < (unsigned)len) && mag_key(xs[k]) >= tau_hat) {
                     const uint2 cv = make_uint2(coord0 + (uint32_t)(r + k), __float_as_uint(xs[k]));
@@ -172,12 +171,13 @@ __global__ void __launch_bounds__(kThreads, 6) topk_sweep_kernel(Tables t, TopkB
     const GT* g = G + row0;
     float* e = b.E + row0;
     const int r0s = ti.r0 - (int)(row0 & 31);
+    const float kept_from = __uint_as_float(b.use_thr ? b.thr[sg] : kNothingKept);
     if (r0s >= 0 && r0s + kTile <= ti.len)
-        topk_sweep_tile<true>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, row0, sh_cand, &sh_cnt,
-                              &st->cand_count, out, cap, b.kept_prev, b.map_words);
+        topk_sweep_tile<true>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
+                              &st->cand_count, out, cap, kept_from);
     else
-        topk_sweep_tile<false>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, row0, sh_cand, &sh_cnt,
-                               &st->cand_count, out, cap, b.kept_prev, b.map_words);
+        topk_sweep_tile<false>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
+                               &st->cand_count, out, cap, kept_from);
     __syncthreads();
     const uint32_t cnt = sh_cnt;
     if (cnt == 0u) return;
@@ -423,6 +423,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     // threshold key of this step (a lower bound if every candidate of the threshold bin is kept)
     const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
     uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
+    // the magnitude from which on everything was kept. With the whole threshold bin kept that is the bin's lower
+    // edge; otherwise the kept candidates of the bin are zeroed in E right here and the next key above the
+    // threshold is left
+    uint32_t kept_from = tau_wide < 0xffffffffull ? (uint32_t)tau_wide : kNothingKept;
+    float* erow = b.E + (size_t)i * (size_t)t.d;
     if (!take_all0) {
         __syncthreads();
         const uint32_t nsurv = sh_scnt;
@@ -466,12 +471,15 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
                 } else {
                     atomicOr(b.status, 1u);
                 }
+                erow[cv.x] = 0.0f;  // the residual of a kept coordinate: e = x - x
             }
             __syncthreads();
         }
         tau = sh_edge[1];
+        kept_from = tau + 1u;
     }
     if (threadIdx.x == 0) {
+        b.thr[sg] = kept_from;
         uint32_t edge;
         if (edge_bin != 0xffffffffu) {
             const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
@@ -696,6 +704,11 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
     }
     const unsigned long long tau_wide = (unsigned long long)tau_hat + ((unsigned long long)b0 << S);
     uint32_t tau = tau_wide < 0x7f7fffffull ? (uint32_t)tau_wide : 0x7f7fffffu;
+    // the magnitude from which on everything was kept. With the whole threshold bin kept that is the bin's lower
+    // edge; otherwise the kept candidates of the bin are zeroed in E right here and the next key above the
+    // threshold is left
+    uint32_t kept_from = tau_wide < 0xffffffffull ? (uint32_t)tau_wide : kNothingKept;
+    float* erow = b.E + (size_t)i * (size_t)t.d;
     if (!take_all0 && nsurv > (uint32_t)kRankMax) {
         // Too many candidates in the threshold bin to rank pair by pair. They differ in the low S key
         // bits and the index; the k_rem-th largest of these (low bits, lower index first) composites
@@ -741,6 +754,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
         // `prefix` is now the composite of the k_rem-th largest candidate (composites are distinct)
         const unsigned long long thr = prefix;
         tau = tau_hat + (uint32_t)(((unsigned long long)b0 << S) | (thr >> 32));
+        kept_from = tau + 1u;
         __syncthreads();
         if (threadIdx.x == 0) {
             sh_base = atomicAdd(&st->emit_count, k_rem);
@@ -757,6 +771,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
                 } else {
                     atomicOr(b.status, 1u);
                 }
+                erow[cv.x] = 0.0f;  // the residual of a kept coordinate: e = x - x
             }
         }
         __syncthreads();
@@ -794,12 +809,15 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
                 } else {
                     atomicOr(b.status, 1u);
                 }
+                erow[cv.x] = 0.0f;  // the residual of a kept coordinate: e = x - x
             }
             __syncthreads();
         }
         tau = sh_tau;
+        kept_from = tau + 1u;
     }
     if (threadIdx.x == 0) {
+        b.thr[sg] = kept_from;
         uint32_t edge;
         if (edge_bin != 0xffffffffu) {
             const unsigned long long ew = (unsigned long long)tau_hat + ((unsigned long long)edge_bin << S);
@@ -894,6 +912,9 @@ __device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b
                 st->prefix = np;
                 st->k_rem = nk;
                 if (PASS == 3) {
+                    // every key above np is kept, and the ties at np too unless only some fit: then the walk over
+                    // the ties zeroes in E the ones it takes and everything from the next key up counts as kept
+                    b.thr[sg] = (nk < cnt[j]) ? np + 1u : np;
                     st->tau = np;
                     st->ties_total = cnt[j];
                     st->ties_take = nk;
@@ -1010,7 +1031,7 @@ __device__ __forceinline__ void dense_ties(const Tables& t, const TopkBuffers& b
     const int tile0 = si->tile0, tile_end = si->tile0 + si->ntile_b;
     const int64_t o = si->o;
     const int len = si->len;
-    const float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
+    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)o;
     const size_t slot0 = (size_t)i * (size_t)b.K + (size_t)si->slot0;
     uint32_t taken = 0;  // ties already assigned to earlier tiles (uniform across the CTA)
     for (int tb = tile0; tb < tile_end && taken < want; tb += kThreads) {
@@ -1046,6 +1067,7 @@ __device__ __forceinline__ void dense_ties(const Tables& t, const TopkBuffers& b
                     b.idx[slot0 + pos] = (int32_t)(o + r);
                     b.val[slot0 + pos] = e[r];
                 }
+                e[r] = 0.0f;  // the residual of a kept coordinate: e = x - x (this thread alone reads and writes e[r])
                 ++rank;
             }
             __syncthreads();
@@ -1204,14 +1226,11 @@ __global__ void __launch_bounds__(kThreads) topk_small_kernel(Tables t, TopkBuff
 }
 
 // ------------------------------------------------------------------------------------------
-// scatter: the kept (index, value) pairs of the messages are handed to the server grouped by coordinate
-// range, and the kept coordinates recorded for the residual update.
+// scatter: the kept (index, value) pairs of the messages are handed to the server grouped by coordinate range.
 
-// All messages at once (`count` pairs of every worker the server averages over; E and the kept map hold
-// the t.n workers of this handle, whose first is worker row0). The first n * nseg threads also close the
-// step for one large-block segment each.
-__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count, int32_t row0,
-                                                                int close) {
+// All messages at once: `count` pairs of every worker the server averages over. The first n * nseg threads also
+// close the step for one large-block segment each when `close` is set (Top-k; Random-k has no selection to close).
+__global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBuffers b, int64_t count, int close) {
     dependency_wait();
     allow_dependents();
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -1223,22 +1242,19 @@ __global__ void __launch_bounds__(kThreads) topk_scatter_kernel(Tables t, TopkBu
         j = __ldg(b.idx + p);
         xbits = __float_as_uint(__ldg(b.val + p));
     }
-    scatter_warp(t, b, valid, j, xbits, valid ? p / b.K - row0 : -1);
+    scatter_warp(b, valid, j, xbits);
 }
 
-// E holds x at the coordinates kept in the last step: zero them (Algorithm 2, the residual update), one thread per word.
-__global__ void __launch_bounds__(kThreads) topk_materialize_kernel(int64_t nd, int64_t map_words,
-                                                                    const uint32_t* __restrict__ kept,
-                                                                    float* __restrict__ E) {
-    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= map_words) return;
-    uint32_t w = kept[q];
-    float* e = E + (size_t)q * 32;
-    while (w) {
-        const int k = __ffs(w) - 1;
-        w &= w - 1;
-        if (q * 32 + k < nd) e[k] = 0.0f;
-    }
+// E holds x at the coordinates kept in the last step: zero them (Algorithm 2, the residual update). One CTA per
+// (tile, worker); the kept elements of a segment are those whose magnitude reaches what its selection left.
+__global__ void __launch_bounds__(kThreads) topk_materialize_kernel(Tables t, TopkBuffers b) {
+    const int i = blockIdx.y;
+    const TileInfo ti = load_tile(t.tiles, blockIdx.x);
+    const float kept_from = __uint_as_float(b.thr[(size_t)i * t.nseg + ti.seg]);
+    float* e = b.E + (size_t)i * (size_t)t.d + (size_t)ti.o;
+    const int end = (ti.r0 + kTile < ti.len) ? ti.r0 + kTile : ti.len;
+    for (int r = ti.r0 + (int)threadIdx.x; r < end; r += kThreads)
+        if (fabsf(e[r]) >= kept_from) e[r] = 0.0f;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1318,9 +1334,8 @@ cudaError_t launch_topk_dense(compams_context* c) {
 }
 
 cudaError_t launch_topk_materialize(compams_context* c) {
-    const int64_t words = c->tk.map_words;
-    topk_materialize_kernel<<<(unsigned)((words + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
-        (int64_t)c->n * c->d, c->tk.map_words, c->keptmap[c->map_cur], c->E);
+    dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
+    topk_materialize_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk);
     return counted(c, cudaGetLastError());
 }
 
@@ -1330,9 +1345,9 @@ cudaError_t launch_topk_scatter(compams_context* c, bool close) {
     const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
     // (a sharded handle's exchange sits in front of this kernel: a plain launch waits for it)
     if (c->chain && c->n == c->n_total)
-        return counted(c, launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count, c->row0,
+        return counted(c, launch_after(topk_scatter_kernel, dim3(grid), dim3(kThreads), c->stream, c->tab, c->tk, count,
                                        close ? 1 : 0));
-    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, c->row0, close ? 1 : 0);
+    topk_scatter_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, count, close ? 1 : 0);
     return counted(c, cudaGetLastError());
 }
 
