@@ -264,18 +264,54 @@ __global__ void __launch_bounds__(kThreads) bs_materialize_kernel(Tables t, floa
     }
 }
 
-constexpr int kApplyChunk = 64;  // workers whose sign words are staged in shared memory at a time
+constexpr int kApplyChunk = 32;  // workers whose sign words are staged (and transposed) at a time: one per lane
+#ifndef COMPAMS_APPLY_TABLES_FROM
+#define COMPAMS_APPLY_TABLES_FROM 20
+#endif
+constexpr int kApplyTablesFrom = COMPAMS_APPLY_TABLES_FROM;  // workers from which the table form of bs_apply is used
 
-// Server side of Block-Sign (Algorithm 2, the server's average and update): one CTA per 1024 consecutive coordinates of a
-// block, one float4 group per thread. The tile's block comes from the constant bank, so the sign
-// words, the scales and the optimizer state are all requested at once. Per coordinate the sum over
-// workers of +-s_i is formed as (sum of all s_i) - 2 (sum of the s_i whose bit is set): one
-// predicated binary64 add per worker, and exact wherever the plain sum is.
+// Transposes four 32 x 32 bit matrices held across a warp: on entry lane i holds x[q] = row i of matrix q
+// (bit c = element (i, c)); on return lane c holds column c (bit i = element (i, c)). Five rounds of the
+// usual block swap: in round j a lane exchanges with lane ^ j the half of its bits whose position differs
+// from its own index in bit j. Shifting the partner's word by +-j and keeping only the positions that
+// change is a rotation followed by a bitwise select.
+__device__ __forceinline__ void transpose32x4(uint32_t (&x)[4], int lane) {
+#pragma unroll
+    for (int j = 16; j >= 1; j >>= 1) {
+        const uint32_t m = j == 16 ? 0x0000ffffu : j == 8 ? 0x00ff00ffu : j == 4 ? 0x0f0f0f0fu : j == 2 ? 0x33333333u : 0x55555555u;
+        const bool up = (lane & j) != 0;
+        const uint32_t keep = up ? ~m : m;          // positions whose bit j equals the lane's stay
+        const uint32_t rot = up ? 32u - j : (uint32_t)j;  // the partner's bits move down (up) by j
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t y = __shfl_xor_sync(0xffffffffu, x[q], j);
+            x[q] = (x[q] & keep) | (__funnelshift_l(y, y, rot) & ~keep);
+        }
+    }
+}
+
+// Server side of Block-Sign (Algorithm 2, the server's average and update): one CTA per 1024 consecutive
+// coordinates of a block, one float4 group per thread. The tile's block comes from the constant bank, so the
+// sign words, the scales and the optimizer state are all requested at once.
+//
+// Per coordinate the sum over workers of +-s_i is (sum of all s_i) - 2 (sum of the s_i whose bit is set).
+// TABLES = false (few workers): one predicated binary64 add per worker and coordinate.
+// TABLES = true: the second sum depends only on the coordinate's pattern of sign bits over the workers, and all
+// 1024 coordinates of the CTA share the workers' scales: for every 4 workers a 16-entry table holds the sum of
+// each subset of their scales (exact in binary64 wherever the plain sum is), and a coordinate adds one table entry
+// per 4 workers instead of testing one bit per worker. The patterns come from transposing the sign words in the
+// warp: lane i reads worker i's four words of the warp's 128 coordinates, transpose32x4 turns them into one word
+// per coordinate, and 16 shuffles hand every lane the patterns of its own 4 coordinates. Up to 32 workers per
+// round. The kernel is bound by instruction issue: the fixed cost of the transposition (36 shuffles per round)
+// pays from about two dozen workers up (n = 32, d = 2^27: step 9.23 -> 8.87 ms; n = 16: no change; n = 8: 3 %
+// slower, hence the two forms).
+template <bool TABLES>
 __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffers b, float* __restrict__ theta,
                                                                HyperParams hp,
                                                                const __grid_constant__ SegParams sp_) {
-    __shared__ uint32_t sh_bits[kApplyChunk][32];
-    __shared__ double sh_s[kApplyChunk];
+    __shared__ uint32_t sh_bits[kApplyChunk][33];        // [worker][word], rows padded against bank conflicts
+    __shared__ double sh_tab[kApplyChunk / 4][16];       // TABLES: [group of 4 workers][subset] sum of the subset's
+                                                         // scales; else: the workers' scales
     const int tile = blockIdx.x >> 3;
     const TileInfo ti = sp_.nseg ? find_tile(sp_, tile) : load_tile(t.tiles, tile);
     const int blk = ti.blk;
@@ -299,27 +335,70 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
         tt = load4(th + r, cls);
     }
     dependency_wait();  // the state above was last written a step ago; sign words and scales are this step's
-    const int wsel = threadIdx.x >> 3, nsh = (threadIdx.x & 7) * 4;
     const size_t wbase = (size_t)(sp_.nseg ? (int64_t)sp_.wofs[ti.seg] : b.word_off[blk]) + (size_t)(rs >> 5);
-    const int wl = threadIdx.x & 31, wr = threadIdx.x >> 5;  // word and worker this thread stages
-    const bool word_live = rs + wl * 32 < len;
+    const int lane = threadIdx.x & 31, wr = threadIdx.x >> 5;  // warp wr owns coordinates 128 wr ... of the CTA's 1024
+    const bool word_live = rs + lane * 32 < len;
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0, all = 0.0;
     for (int i0 = 0; i0 < t.n; i0 += kApplyChunk) {
         const int nc = (t.n - i0 < kApplyChunk) ? t.n - i0 : kApplyChunk;
         __syncthreads();
+        // warp wr stages the words of workers wr, wr + 8, ...: 32 consecutive words each, one per lane
         for (int c = wr; c < nc; c += kWarps)
-            sh_bits[c][wl] = word_live ? __ldg(b.bits + (size_t)(i0 + c) * (size_t)b.W + wbase + wl) : 0u;
-        if (threadIdx.x < nc) sh_s[threadIdx.x] = (double)b.scales_cur[(size_t)(i0 + threadIdx.x) * t.M + blk];
-        __syncthreads();
+            sh_bits[c][lane] = word_live ? __ldg(b.bits + (size_t)(i0 + c) * (size_t)b.W + wbase + lane) : 0u;
+        if constexpr (TABLES) {
+            const int ng = (nc + 3) >> 2;  // groups of 4 workers in this round
+            if (threadIdx.x < ng * 16) {   // one table entry per thread: the scales of the subset's members
+                const int gq = threadIdx.x >> 4, sub = threadIdx.x & 15;
+                double e = 0.0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (((sub >> j) & 1) && gq * 4 + j < nc)
+                        e += (double)b.scales_cur[(size_t)(i0 + gq * 4 + j) * t.M + blk];
+                sh_tab[gq][sub] = e;
+            }
+            __syncthreads();
+            // lane i: worker i's words of this warp's coordinates -> lane c: the workers' bits of coordinate 32 q + c
+            uint32_t x[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) x[q] = lane < nc ? sh_bits[lane][wr * 4 + q] : 0u;
+            transpose32x4(x, lane);
+            // this thread's coordinates 4 lane + k lie in word q = lane / 8 at bit 4 (lane % 8) + k: their patterns
+            // sit in lane 4 (lane % 8) + k, matrix lane / 8 (a trip through shared memory instead of these 16
+            // shuffles was slower)
+            uint4 pat = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t y0 = __shfl_sync(0xffffffffu, x[q], (lane & 7) * 4 + 0);
+                const uint32_t y1 = __shfl_sync(0xffffffffu, x[q], (lane & 7) * 4 + 1);
+                const uint32_t y2 = __shfl_sync(0xffffffffu, x[q], (lane & 7) * 4 + 2);
+                const uint32_t y3 = __shfl_sync(0xffffffffu, x[q], (lane & 7) * 4 + 3);
+                if ((lane >> 3) == q) pat = make_uint4(y0, y1, y2, y3);
+            }
+#pragma unroll
+            for (int gq = 0; gq < kApplyChunk / 4; ++gq) {
+                if (gq < ng) {  // the same for every thread of the CTA
+                    all += sh_tab[gq][15];
+                    a0 += sh_tab[gq][(pat.x >> (4 * gq)) & 15u];
+                    a1 += sh_tab[gq][(pat.y >> (4 * gq)) & 15u];
+                    a2 += sh_tab[gq][(pat.z >> (4 * gq)) & 15u];
+                    a3 += sh_tab[gq][(pat.w >> (4 * gq)) & 15u];
+                }
+            }
+        } else {
+            double* sh_s = &sh_tab[0][0];
+            if (threadIdx.x < nc) sh_s[threadIdx.x] = (double)b.scales_cur[(size_t)(i0 + threadIdx.x) * t.M + blk];
+            __syncthreads();
+            const int wsel = threadIdx.x >> 3, nsh = (threadIdx.x & 7) * 4;  // this thread's word and its nibble in it
 #pragma unroll 4
-        for (int c = 0; c < nc; ++c) {
-            const double s = sh_s[c];
-            const uint32_t nib = sh_bits[c][wsel] >> nsh;
-            all += s;
-            if (nib & 1u) a0 += s;
-            if (nib & 2u) a1 += s;
-            if (nib & 4u) a2 += s;
-            if (nib & 8u) a3 += s;
+            for (int c = 0; c < nc; ++c) {
+                const double sc = sh_s[c];
+                const uint32_t nib = sh_bits[c][wsel] >> nsh;
+                all += sc;
+                if (nib & 1u) a0 += sc;
+                if (nib & 2u) a1 += sc;
+                if (nib & 4u) a2 += sc;
+                if (nib & 8u) a3 += sc;
+            }
         }
     }
     a0 = all - (a0 + a0);
@@ -395,11 +474,16 @@ cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     Tables t = c->tab;
     t.n = c->n_total;  // the average runs over every worker's message
     const dim3 grid((unsigned)c->tab.ntiles * kWarps);
+    const bool tables = c->n_total >= kApplyTablesFrom;
     if (c->n == c->n_total)
-        return counted(c, launch_after(bs_apply_kernel, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp));
+        return counted(c, tables ? launch_after(bs_apply_kernel<true>, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp)
+                                 : launch_after(bs_apply_kernel<false>, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp));
     // sharded workers: the other workers' messages were written by the caller's exchange, which is
     // ordered on the stream like any kernel; a plain launch waits for it
-    bs_apply_kernel<<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
+    if (tables)
+        bs_apply_kernel<true><<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
+    else
+        bs_apply_kernel<false><<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
     return counted(c, cudaGetLastError());
 }
 

@@ -146,11 +146,67 @@ __device__ __forceinline__ void topk_sweep_tile(const GT* __restrict__ g, float*
     }
 }
 
+// The same for bfloat16 gradients on a whole tile whose rows of G and E are 16-byte aligned: 8 coordinates per
+// lane and iteration, so that the gradient load is 128 bits wide like the loads and stores of E (with 4
+// coordinates per lane the 64-bit gradient loads leave too few bytes in flight). A warp's 1024 coordinates are
+// 4 chunks of 256; the next chunk's loads are in flight while one is worked on.
+__device__ __forceinline__ void topk_sweep_tile_bf16x8(const bf16_bits* __restrict__ g, float* __restrict__ e, int r0,
+                                                       int warp, int lane, uint32_t tau_hat, uint32_t coord0,
+                                                       uint2* sh_cand, uint32_t* sh_cnt, uint32_t* g_cnt, uint2* g_out,
+                                                       uint32_t cap, float kept_from) {
+    constexpr int NC = kWarpSpan / 256;
+    const int rw = r0 + warp * kWarpSpan;
+    uint4 gbuf[2];
+    float4 ebuf[2][2];
+    auto load_chunk = [&](int c, uint4& gv, float4 (&ev)[2]) {
+        const int r = rw + c * 256 + lane * 8;
+        gv = __ldg(reinterpret_cast<const uint4*>(g + r));
+        ev[0] = *reinterpret_cast<const float4*>(e + r);
+        ev[1] = *reinterpret_cast<const float4*>(e + r + 4);
+    };
+    load_chunk(0, gbuf[0], ebuf[0]);
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const uint4 gv = gbuf[c & 1];
+        float4 (&ev)[2] = ebuf[c & 1];
+        if (c + 1 < NC) load_chunk(c + 1, gbuf[(c + 1) & 1], ebuf[(c + 1) & 1]);
+        const int r = rw + c * 256 + lane * 8;
+        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float xs[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t word = gw[h * 2 + (k >> 1)];
+                const float gk = __uint_as_float((k & 1) ? (word & 0xffff0000u) : (word << 16));  // exact widening
+                // coordinates kept in the last step still hold x in E: their e is 0 (Algorithm 2, the residual update)
+                const float eo = lane_elem(ev[h], k);
+                const float ek = fabsf(eo) >= kept_from ? 0.0f : eo;
+                xs[k] = __fadd_rn(gk, ek);  // the corrected-gradient step: x = g + e
+                if (mag_key(xs[k]) >= tau_hat) {
+                    const uint2 cv = make_uint2(coord0 + (uint32_t)(r + h * 4 + k), __float_as_uint(xs[k]));
+                    const uint32_t slot = atomicAdd(sh_cnt, 1u);
+                    if (slot < (uint32_t)kTileCand) {
+                        sh_cand[slot] = cv;
+                    } else {  // a tile dense with candidates: the staging buffer is full, append directly
+                        const uint32_t p = atomicAdd(g_cnt, 1u);
+                        if (p < cap) g_out[p] = cv;
+                    }
+                }
+            }
+            *reinterpret_cast<float4*>(e + r + h * 4) = make_float4(xs[0], xs[1], xs[2], xs[3]);
+        }
+    }
+}
+
 // Tiles are shifted down by (i d + o) mod 32, the position of the block's first element within a
 // 128-byte line of G and E, so that every warp access covers whole lines (with rows that start
 // mid-line a warp's 512 bytes straddle five lines instead of four: measured 7 % slower).
+#ifndef COMPAMS_BF16_TOPK_SWEEP_CTAS
+#define COMPAMS_BF16_TOPK_SWEEP_CTAS 5
+#endif
 template <typename GT>
-__global__ void __launch_bounds__(kThreads, 6) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
+__global__ void __launch_bounds__(kThreads, sizeof(GT) == 2 ? COMPAMS_BF16_TOPK_SWEEP_CTAS : 6) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
                                                                  const __grid_constant__ SegParams sp_) {
     dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
@@ -172,7 +228,15 @@ __global__ void __launch_bounds__(kThreads, 6) topk_sweep_kernel(Tables t, TopkB
     float* e = b.E + row0;
     const int r0s = ti.r0 - (int)(row0 & 31);
     const float kept_from = __uint_as_float(b.use_thr ? b.thr[sg] : kNothingKept);
-    if (r0s >= 0 && r0s + kTile <= ti.len)
+    const bool whole = r0s >= 0 && r0s + kTile <= ti.len;
+    bool wide = false;
+    if constexpr (sizeof(GT) == 2)
+        wide = whole && ((reinterpret_cast<uintptr_t>(g + r0s) | reinterpret_cast<uintptr_t>(e + r0s)) & 15u) == 0;
+    if (wide) {
+        if constexpr (sizeof(GT) == 2)
+            topk_sweep_tile_bf16x8(g, e, r0s, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt, &st->cand_count, out,
+                                   cap, kept_from);
+    } else if (whole)
         topk_sweep_tile<true>(g, e, ti.len, r0s, warp, lane, tau_hat, (uint32_t)ti.o, sh_cand, &sh_cnt,
                               &st->cand_count, out, cap, kept_from);
     else

@@ -51,6 +51,14 @@ def test_blocksign_ragged_blocks(n, check_e_every):
     _pair_run(n, d, RAGGED, BLOCKSIGN, 1.0, _randn(n, d), steps=5, check_e_every=check_e_every)
 
 
+@pytest.mark.parametrize("n", [2, 7, 31, 32, 33, 70])
+def test_blocksign_worker_counts_around_the_transposition_width(n):
+    # the server kernel transposes the sign words of up to 32 workers at a time and looks up the scales of 4
+    # workers at once: worker counts below, at and above those widths, blocks that end inside a word
+    d = 2 * 8192 + 1234
+    _pair_run(n, d, [0, 37, 5000, 8192 + 100, d], BLOCKSIGN, 1.0, _randn(n, d), steps=3)
+
+
 @pytest.mark.parametrize("d", [1, 2, 3, 5, 31, 33, 4096, 4097, 8191, 8192, 8193, 3 * 8192 + 2])
 @pytest.mark.parametrize("comp", [TOPK, BLOCKSIGN])
 def test_single_block_sizes_around_tile_edges(d, comp):

@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2205_05632_b200 import BLOCKSIGN, TOPK, CompAMS, CompAMSError
+from paper_2205_05632_b200 import BLOCKSIGN, RANDK, TOPK, CompAMS, CompAMSError
 
 pytestmark = pytest.mark.gpu
 
@@ -66,7 +66,7 @@ def _run(comp, ratio, offs, n_total, R, steps=5, seed=0):
         o.close()
 
 
-@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (TOPK, 0.2), (BLOCKSIGN, 1.0)])
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (TOPK, 0.2), (BLOCKSIGN, 1.0), (RANDK, 0.05)])
 @pytest.mark.parametrize("n_total,R", [(4, 2), (6, 3), (4, 4)])
 def test_shards_reproduce_the_whole_layerwise(comp, ratio, n_total, R):
     _run(comp, ratio, OFFS, n_total, R)
