@@ -473,6 +473,47 @@ def test_calls_out_of_order_are_rejected():
         ref.close()
 
 
+# ------------------------------------------------------------------ randomised shapes and value distributions
+
+@pytest.mark.parametrize("seed", range(30))
+def test_randomised_partitions_ratios_and_distributions(seed):
+    # random block partitions (tiny, small and tiled blocks mixed), worker counts, keep ratios and gradient
+    # distributions that change from step to step - continuous, heavy-tailed, quantised to a few levels (ties at
+    # the threshold, kept and cut), exact zeros, scale jumps - for the three compressors, every step against the
+    # oracle; reading E on some steps only exercises the deferred residual on the others
+    rng = np.random.default_rng(1000 + seed)
+    n = int(rng.choice([1, 2, 3, 5, 8]))
+    sizes = []
+    for _ in range(int(rng.integers(1, 9))):
+        kind = rng.integers(0, 4)
+        sizes.append(int(rng.integers(1, 40)) if kind == 0 else int(rng.integers(40, 4097)) if kind == 1
+                     else int(rng.integers(4097, 30000)) if kind == 2 else int(rng.integers(30000, 120000)))
+    offs = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    d = offs[-1]
+    comp = [TOPK, BLOCKSIGN, RANDK][seed % 3]
+    ratio = float(rng.choice([0.001, 0.01, 0.05, 0.3]))
+    kinds = rng.integers(0, 5, size=8)
+    scales = 10.0 ** rng.integers(-3, 3, size=8)
+
+    def make(gen, t):
+        kind, sc = int(kinds[t]), float(scales[t]) if t % 3 == 2 else 1.0
+        if kind == 0:
+            g = torch.randn(n, d, generator=gen, device="cuda")
+        elif kind == 1:
+            z = torch.randn(2, n, d, generator=gen, device="cuda")
+            g = z[0] / z[1].abs().clamp_min(1e-3)                      # heavy tails
+        elif kind == 2:
+            g = torch.randint(-3, 4, (n, d), generator=gen, device="cuda").float()   # seven levels: ties everywhere
+        elif kind == 3:
+            g = torch.randn(n, d, generator=gen, device="cuda")
+            g[torch.rand(n, d, generator=gen, device="cuda") < 0.5] = 0.0  # half exact zeros
+        else:
+            g = torch.randint(-40, 41, (n, d), generator=gen, device="cuda").float() * 0.25
+        return g * sc
+
+    _pair_run(n, d, offs, comp, ratio, make, steps=8, check_e_every=3)
+
+
 # ------------------------------------------------------------------ Random-k
 
 @pytest.mark.parametrize("n", [1, 3])
