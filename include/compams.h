@@ -312,9 +312,10 @@ int compams_bits_transmitted(compams_handle h, uint64_t* out);
  * The contents are those of the last enqueued step once the stream has reached that point;
  * they stay valid until the next compams_step / compams_destroy. Asking for BUF_E enqueues
  * one extra kernel that finishes the residual update of Algorithm 2 in place: the step itself leaves the
- * corrected gradient x in E (Block-Sign: all of it; Top-k: at the kept coordinates, which are
- * recorded in a bit map) and applies e = x - g~ when E is next read, by the next iteration's sweep
- * or by this call; the values are identical either way.
+ * corrected gradient x in E (Block-Sign: all of it; Top-k: at the kept coordinates, which are the
+ * ones whose magnitude reaches a value the selection leaves per worker and block) and applies
+ * e = x - g~ when E is next read, by the next iteration's sweep or by this call; the values are
+ * identical either way. (Random-k zeroes its kept coordinates at once.)
  *
  * SIGN_BITS layout: row i has W words; block b starts at word SIGN_WORD_OFFSETS[b]; bit (r % 32)
  * of word SIGN_WORD_OFFSETS[b] + r / 32 is the sign bit of x at coordinate block_offsets[b] + r;
