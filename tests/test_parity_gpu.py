@@ -565,6 +565,47 @@ def test_randk_sets_follow_seed_and_iteration_count():
     assert torch.equal(a[1], late[0]) and torch.equal(a[2], late[1])  # iteration t + 1 of one run = iteration t of a run started one later
 
 
+# ------------------------------------------------------------------ streams
+
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (BLOCKSIGN, 1.0), (RANDK, 0.01), (TOPK, 1.0)])
+def test_steps_on_a_side_stream_match_the_default_stream(comp, ratio):
+    # everything a step enqueues - programmatic dependents, the cooperative dense-pass kernel, the host-buffer
+    # copies - goes to the handle's stream: a handle on a side stream, fed by producers on that stream, must give
+    # the bits of a handle on the default stream; moving a handle to another stream (ordered by an event) too
+    n, d = 3, 6 * 8192 + 321
+    offs = [0, 3000, 30000, d]
+    gen = torch.Generator(device="cuda").manual_seed(12)
+    G = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(5)]
+    ref = CompAMS(n, d, offs, comp, ratio)
+    theta_ref = torch.zeros(d, device="cuda")
+    for g in G:
+        ref.step(g, theta_ref)
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    theta = torch.zeros(d, device="cuda")
+    with torch.cuda.stream(s1):
+        opt = CompAMS(n, d, offs, comp, ratio, stream=s1)
+        for g in G[:3]:
+            staged = g.clone()          # produced on s1, consumed by the step on s1
+            opt.step(staged, theta)
+        done = torch.cuda.Event()
+        done.record(s1)
+    s2.wait_event(done)
+    opt.set_stream(s2)
+    with torch.cuda.stream(s2):
+        for g in G[3:]:
+            opt.step(g.clone(), theta)
+        e_side = opt.buffer("E").clone()
+    s2.synchronize()
+    assert opt.check_status() == 0
+    assert torch.equal(theta, theta_ref)
+    assert torch.equal(e_side, ref.buffer("E"))
+    for name in ("m", "v", "vhat", "gbar"):
+        assert torch.equal(opt.buffer(name), ref.buffer(name)), name
+    opt.close()
+    ref.close()
+
+
 # ------------------------------------------------------------------ checkpoint / restore, traffic accounting
 
 @pytest.mark.parametrize("comp,ratio", [(TOPK, 0.02), (BLOCKSIGN, 1.0), (TOPK, 1.0)])
