@@ -144,7 +144,7 @@ int compams_step(compams_handle h, const float* grads, float* theta);
 /*
  * compams_step_bf16 / compams_compress_bf16 - compams_step / compams_compress for gradients stored as
  * bfloat16 (what a mixed-precision backward pass produces): the worker-side read of g shrinks from 4 to
- * 2 bytes per element, everything else is unchanged. Line 7 of Algorithm 2 becomes x = widen(g) + e with
+ * 2 bytes per element, everything else is unchanged. The corrected-gradient step of Algorithm 2 becomes x = widen(g) + e with
  * widen exact, so the step equals compams_step on the fp32 tensor that holds the same values, bit for bit;
  * e, the messages and the server state stay fp32. A handle may be fed fp32 in one step and bfloat16 in
  * the next.
