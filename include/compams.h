@@ -138,6 +138,13 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
  * coordinate plus one scale per (worker, block). sign(x) follows the IEEE sign bit (+0 -> +,
  * -0 -> -), so every coordinate of a block contributes exactly +-scale.
  * Errors: INVALID_ARG (null or misaligned pointer), CUDA (launch failure).
+ *
+ * A step enqueues kernels only (no allocation, no host synchronisation), so it may be captured into a CUDA
+ * graph on the handle's stream. What the captured launches bake in are the handle's host-side switches of
+ * that moment (which of two alternating buffers is current, whether E still holds the last step's x): they
+ * repeat with period two once one step has run, so capture an even number of steps after a first eager
+ * step, and refill the captured gradient buffers before every replay. Not for COMPAMS_RANDK (the iteration
+ * index that keys its index sets is a kernel argument); compams_bits_transmitted counts captured steps once.
  */
 int compams_step(compams_handle h, const float* grads, float* theta);
 
