@@ -20,13 +20,13 @@ from typing import Iterable, List
 import numpy as np
 import torch
 
-from .binding import TOPK, CompAMS, CompAMSError
+from .binding import RANDK, TOPK, CompAMS, CompAMSError
 
 
 class CompAMSOptimizer:
     def __init__(self, params: Iterable[torch.nn.Parameter], n_workers: int, compressor: int = TOPK,
                  k_ratio: float = 0.01, whole_vector: bool = False, lr: float = 1e-3, beta1: float = 0.9,
-                 beta2: float = 0.999, eps: float = 1e-8):
+                 beta2: float = 0.999, eps: float = 1e-8, seed: int = 0):
         self.params: List[torch.nn.Parameter] = [p for p in params if p.requires_grad]
         if not self.params:
             raise CompAMSError("no trainable parameters")
@@ -46,6 +46,8 @@ class CompAMSOptimizer:
         blocks = np.array([0, self.d], dtype=np.int64) if whole_vector else self.offsets
         with torch.cuda.device(dev):
             self.opt = CompAMS(self.n, self.d, blocks, compressor, k_ratio, lr, beta1, beta2, eps)
+            if compressor == RANDK:
+                self.opt.set_seed(seed)  # Random-k: the seed of the index sets
 
     def collect(self, worker: int) -> None:
         """Row `worker` of G <- the gradients accumulated since the last collect(); they are cleared."""

@@ -65,7 +65,7 @@ def test_single_block_sizes_around_tile_edges(d, comp):
     _pair_run(2, d, [0, d], comp, 0.1, _randn(2, d), steps=3)
 
 
-@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (TOPK, 0.3), (TOPK, 1.0), (BLOCKSIGN, 1.0)])
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (TOPK, 0.3), (TOPK, 1.0), (BLOCKSIGN, 1.0), (RANDK, 0.05)])
 @pytest.mark.parametrize("n", [1, 3, 4])
 def test_bfloat16_gradients_ragged_blocks(comp, ratio, n):
     # d = 3 mod 4 and odd block offsets: rows and blocks of the bfloat16 tensor start in every alignment class
