@@ -189,6 +189,13 @@ def workload_config(pt):
     }
 
 
+def _as_randk(w):
+    """The same workload compressed with Random-k instead of Top-k."""
+    w.compressor = W.RANDK
+    w.name = w.name.replace("C3", "C3/randk")
+    return w
+
+
 def config_entries():
     """Every timed entry of "configs": (name, builder of the workload on a device, mode, bfloat16 input)."""
     out = [("C1/topk1%", lambda dev: W.config1(dev), "topk", False),
@@ -199,6 +206,7 @@ def config_entries():
            ("C3/topk1%/bf16", lambda dev: W.config3(0.01, dev), "topk", True),
            ("C4/topk1%/layerwise", lambda dev: W.config4(W.TOPK, dev), "topk", False),
            ("C4/sign", lambda dev: W.config4(W.BLOCKSIGN, dev), "sign", False)]
+    out.append(("C3/randk1%", lambda dev: _as_randk(W.config3(0.01, dev)), "randk", False))
     for lg in (20, 22, 24, 26, 27):
         for n in (1, 8, 32):
             for mode in ("topk", "sign", "dense"):

@@ -263,10 +263,12 @@ int compams_set_stream(compams_handle h, void* cuda_stream);
  * The drawing rule (Section 2.1 only names Random-k; this is the library's reading, fixed so that a
  * second implementation can reproduce the sets bit for bit): worker i keeps in block b, at iteration t,
  * the coordinates block_offsets[b] + pi(r), r = 0 .. k_b - 1, where pi is a permutation of {0 .. d_b - 1}:
- * a balanced Feistel network of four rounds over the smallest even number of bits 2w with 2^(2w) >= d_b
- * (at least 2), applied again while the result is >= d_b. Round `round` maps (L, R) to (R, L xor (F & (2^w - 1)))
- * with F the first output word of Philox4x64-10 (Salmon et al., SC 2011) at counter (R, round, b, i) under
- * key (seed, t); the input is L = r >> w, R = r & (2^w - 1), the output (L << w) | R. Workers are numbered
+ * a balanced Feistel network of six rounds over the smallest even number of bits 2w with 2^(2w) >= d_b
+ * (at least 2), applied again while the result is >= d_b. Round r maps (L, R) to
+ * (R, L xor (F(R xor key_r) & (2^w - 1))): F is the 32-bit finalizer of MurmurHash3 (h ^= h >> 16;
+ * h *= 0x85ebca6b; h ^= h >> 13; h *= 0xc2b2ae35; h ^= h >> 16) and key_0 .. key_5 are the low and high
+ * 32-bit halves of the first three output words of Philox4x64-10 (Salmon et al., SC 2011) at counter
+ * (0, 0, b, i) under key (seed, t); the input is L = r >> w, R = r & (2^w - 1), the output (L << w) | R. Workers are numbered
  * over the whole job (first_worker + local index on a sharded handle).
  */
 int compams_set_seed(compams_handle h, uint64_t seed, uint64_t iterations_done);

@@ -119,25 +119,41 @@ void philox4x64_10(const uint64_t ctr[4], const uint64_t key[2], uint64_t out[4]
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-// A keyed pseudorandom permutation of {0, ..., m-1}: a balanced Feistel network of four rounds over the
-// smallest even number of bits 2w with 2^(2w) >= m (at least 2), whose round function is the first word
-// of Philox4x64-10 at counter (right half, round, block, worker) under key (seed, step); a result
-// outside [0, m) is fed through the network again until it falls inside (cycle walking), which makes the
-// restriction to [0, m) a bijection.
-uint64_t randk_permute(uint64_t m, uint64_t r, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block) {
-    int bits = 2;
-    while (bits < 64 && ((uint64_t)1 << bits) < m) bits += 2;
-    const int w = bits / 2;
-    const uint64_t mask = ((uint64_t)1 << w) - 1;
+// The 32-bit finalizer of MurmurHash3 (Appleby): a bijection of the 32-bit words that mixes every input bit
+// into every output bit.
+inline uint32_t fmix32(uint32_t h) {
+    h ^= h >> 16;
+    h *= 0x85ebca6bu;
+    h ^= h >> 13;
+    h *= 0xc2b2ae35u;
+    h ^= h >> 16;
+    return h;
+}
+
+// The six 32-bit round keys of (seed, step, worker, block): the low and high halves of the first three words
+// of one Philox4x64-10 block at counter (0, 0, block, worker) under key (seed, step).
+void randk_round_keys(uint64_t seed, uint64_t step, uint64_t worker, uint64_t block, uint32_t keys[6]) {
+    const uint64_t ctr[4] = {0, 0, block, worker};
     const uint64_t key[2] = {seed, step};
-    uint64_t x = r;
+    uint64_t w[4];
+    philox4x64_10(ctr, key, w);
+    for (int r = 0; r < 6; ++r) keys[r] = (uint32_t)(r & 1 ? w[r >> 1] >> 32 : w[r >> 1]);
+}
+
+// A keyed pseudorandom permutation of {0, ..., m-1}, m < 2^32: a balanced Feistel network of six rounds over the
+// smallest even number of bits 2w with 2^(2w) >= m (at least 2), round r mapping (L, R) to
+// (R, L xor (fmix32(R xor key_r) mod 2^w)); a result outside [0, m) is fed through the network again until it
+// falls inside (cycle walking), which makes the restriction to [0, m) a bijection.
+uint64_t randk_permute_keyed(uint64_t m, uint64_t r, const uint32_t keys[6]) {
+    int bits = 2;
+    while (bits < 32 && ((uint64_t)1 << bits) < m) bits += 2;
+    const int w = bits / 2;
+    const uint32_t mask = ((uint32_t)1 << w) - 1;
+    uint32_t x = (uint32_t)r;
     do {
-        uint64_t L = x >> w, R = x & mask;
-        for (uint64_t round = 0; round < 4; ++round) {
-            const uint64_t ctr[4] = {R, round, block, worker};
-            uint64_t f[4];
-            philox4x64_10(ctr, key, f);
-            const uint64_t nR = L ^ (f[0] & mask);
+        uint32_t L = x >> w, R = x & mask;
+        for (int round = 0; round < 6; ++round) {
+            const uint32_t nR = L ^ (fmix32(R ^ keys[round]) & mask);
             L = R;
             R = nR;
         }
@@ -146,12 +162,20 @@ uint64_t randk_permute(uint64_t m, uint64_t r, uint64_t seed, uint64_t step, uin
     return x;
 }
 
+uint64_t randk_permute(uint64_t m, uint64_t r, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block) {
+    uint32_t keys[6];
+    randk_round_keys(seed, step, worker, block, keys);
+    return randk_permute_keyed(m, r, keys);
+}
+
 // Random-k on one block of `len` coordinates: the kept set is { pi(r) : r = 0 .. k-1 }, pi the permutation
 // above for this (seed, step, worker, block): k distinct coordinates, every k-subset (nearly) equally
 // likely, the same set whenever the four identifiers are the same. The values play no part.
 void randk_block(int64_t len, int64_t k, uint64_t seed, uint64_t step, uint64_t worker, uint64_t block, uint8_t* keep) {
     std::memset(keep, 0, (size_t)len);
-    for (int64_t r = 0; r < k; ++r) keep[randk_permute((uint64_t)len, (uint64_t)r, seed, step, worker, block)] = 1;
+    uint32_t keys[6];
+    randk_round_keys(seed, step, worker, block, keys);
+    for (int64_t r = 0; r < k; ++r) keep[randk_permute_keyed((uint64_t)len, (uint64_t)r, keys)] = 1;
 }
 
 struct Oracle {

@@ -186,8 +186,8 @@ def config4(compressor: int, device="cpu", n: int = 32) -> Workload:
 
 
 def sweep_point(d: int, n: int, mode: str, device="cpu") -> Workload:
-    """Scaling sweep: one block, gradients N(0,1); mode in {"topk", "sign", "dense"} (dense: k = d)."""
-    comp = BLOCKSIGN if mode == "sign" else TOPK
-    ratio = {"topk": 0.01, "sign": 1.0, "dense": 1.0}[mode]
+    """Scaling sweep: one block, gradients N(0,1); mode in {"topk", "sign", "dense", "randk"} (dense: k = d)."""
+    comp = BLOCKSIGN if mode == "sign" else RANDK if mode == "randk" else TOPK
+    ratio = {"topk": 0.01, "sign": 1.0, "dense": 1.0, "randk": 0.01}[mode]
     return Workload("C5[%s,d=%d,n=%d]" % (mode, d, n), n, d, np.array([0, d], dtype=np.int64), comp, ratio,
                     device=device, _row=_row_normal)

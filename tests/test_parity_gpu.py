@@ -292,7 +292,7 @@ def test_config5_sweep_point_d_2_24_n_8_against_the_full_oracle(mode):
     run_workload(W.sweep_point(1 << 24, 8, mode, "cuda"), steps=10, check_e_every=5)
 
 
-@pytest.mark.parametrize("mode", ["topk", "sign", "dense"])
+@pytest.mark.parametrize("mode", ["topk", "sign", "dense", "randk"])
 def test_config5_largest_point_d_2_27_n_32_against_the_full_oracle(mode):
     # the largest configuration: n d = 2^32 elements (16 GiB per [n, d] buffer), every index beyond 32 bits.
     # Two chained steps: the first Top-k selection runs the dense passes, the second the candidate path.
