@@ -80,55 +80,78 @@ __device__ __forceinline__ uint32_t randk_permute(uint32_t m, uint32_t r, const 
     return x;
 }
 
-// One thread per message slot of this handle's t.n workers (worker il of the handle is worker row0 + il of the
-// job). The slots of one (worker, block) are consecutive, so within a CTA the thread holding a block's first slot
-// (or thread 0, for a block begun in the CTA before) derives the round keys once and the others read them from
-// shared memory.
-__global__ void __launch_bounds__(kThreads) randk_emit_kernel(Tables t, TopkBuffers b, int32_t row0, uint64_t seed,
-                                                              uint64_t step, int deliver) {
-    __shared__ uint32_t keys[kThreads][6];
+struct Drawn {
+    bool valid;
+    int32_t il;  // worker within the handle
+    int64_t q;   // slot within the worker's message row
+    int32_t j;   // the drawn coordinate
+};
+
+// A CTA covers kThreads consecutive message slots of one worker; every thread computes the coordinate of its
+// slot. The slots of one block are consecutive, so the thread holding a block's first slot (or thread 0, for a
+// block begun in the CTA before) derives the round keys once and the others read them from shared memory.
+// Called by all threads of the CTA.
+__device__ __forceinline__ Drawn randk_draw(const Tables& t, const TopkBuffers& b, int32_t row0, uint64_t seed,
+                                            uint64_t step, uint32_t (*keys)[6]) {
+    const uint32_t per_worker = (uint32_t)((b.K + kThreads - 1) / kThreads);
     const int tid = threadIdx.x;
-    const int64_t p = (int64_t)blockIdx.x * blockDim.x + tid;
-    const bool valid = p < (int64_t)t.n * b.K;
-    int64_t il = 0, q = 0, o = 0;
-    int lo = 0;
+    Drawn dr;
+    dr.il = (int32_t)(blockIdx.x / per_worker);
+    dr.q = (int64_t)(blockIdx.x % per_worker) * kThreads + tid;
+    dr.valid = dr.q < b.K;
+    dr.j = 0;
+    int64_t o = 0;
     uint32_t len = 1, r = 0;
-    if (valid) {
-        il = p / b.K;
-        q = p % b.K;  // slot within the worker's row; its block by bisection of the slot offsets
-        int hi = t.M - 1;
+    if (dr.valid) {
+        int lo = 0, hi = t.M - 1;  // the slot's block, by bisection of the slot offsets
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
-            if (__ldg(b.seg_off + mid) <= q) lo = mid; else hi = mid - 1;
+            if (__ldg(b.seg_off + mid) <= dr.q) lo = mid; else hi = mid - 1;
         }
         o = __ldg(t.off + lo);
         len = (uint32_t)(__ldg(t.off + lo + 1) - o);
-        r = (uint32_t)(q - __ldg(b.seg_off + lo));
+        r = (uint32_t)(dr.q - __ldg(b.seg_off + lo));
         if (tid == 0 || r == 0) {
-            const RoundKeys rk = randk_round_keys(seed, step, (uint64_t)(row0 + il), (uint64_t)lo);
+            const RoundKeys rk = randk_round_keys(seed, step, (uint64_t)(row0 + dr.il), (uint64_t)lo);
 #pragma unroll
             for (int i = 0; i < 6; ++i) keys[tid][i] = rk.k[i];
         }
     }
     __syncthreads();
-    int32_t j = 0;
-    uint32_t xbits = 0;
-    if (valid) {
+    if (dr.valid) {
         const int leader = r < (uint32_t)tid ? tid - (int)r : 0;
-        j = (int32_t)(o + randk_permute(len, r, keys[leader]));
-        float* ex = b.E + (size_t)il * (size_t)t.d + (size_t)j;
-        xbits = __float_as_uint(*ex);  // the sweep left x = g + e there
-        *ex = 0.0f;                    // the residual update at a kept coordinate: e = x - x
-        const size_t slot = (size_t)(row0 + il) * (size_t)b.K + (size_t)q;
-        b.idx[slot] = j;
-        b.val[slot] = __uint_as_float(xbits);
+        dr.j = (int32_t)(o + randk_permute(len, r, keys[leader]));
     }
-    if (deliver) scatter_warp(b, valid, j, xbits);
+    return dr;
+}
+
+// Worker il keeps coordinate j in message slot q: x goes to the message, its residual is zero.
+__device__ __forceinline__ uint32_t randk_take(const Tables& t, const TopkBuffers& b, int32_t row0, int32_t il, int64_t q,
+                                               int32_t j) {
+    // the sweep left x = g + e there; the residual of a kept coordinate is e = x - x = 0. One exchange at the L2
+    // fetches the one and leaves the other (a load followed by a store to the same scattered word made this
+    // kernel six times slower).
+    uint32_t* ex = reinterpret_cast<uint32_t*>(b.E + (size_t)il * (size_t)t.d + (size_t)j);
+    const uint32_t xbits = atomicExch(ex, 0u);
+    const size_t slot = (size_t)(row0 + il) * (size_t)b.K + (size_t)q;
+    b.idx[slot] = j;
+    b.val[slot] = __uint_as_float(xbits);
+    return xbits;
+}
+
+// One thread per message slot draws its coordinate and takes it.
+__global__ void __launch_bounds__(kThreads) randk_emit_kernel(Tables t, TopkBuffers b, int32_t row0, uint64_t seed,
+                                                              uint64_t step, int deliver) {
+    __shared__ uint32_t keys[kThreads][6];
+    const Drawn dr = randk_draw(t, b, row0, seed, step, keys);
+    uint32_t xbits = 0;
+    if (dr.valid) xbits = randk_take(t, b, row0, dr.il, dr.q, dr.j);
+    if (deliver) scatter_warp(b, dr.valid, dr.j, xbits);
 }
 
 cudaError_t launch_randk_emit(compams_context* c, bool deliver) {
-    const int64_t count = (int64_t)c->n * c->K;
-    const unsigned grid = (unsigned)((count + kThreads - 1) / kThreads);
+    const int64_t per_worker = (c->K + kThreads - 1) / kThreads;
+    const unsigned grid = (unsigned)(per_worker * c->n);
     randk_emit_kernel<<<grid, kThreads, 0, c->stream>>>(c->tab, c->tk, c->row0, c->seed, c->iter, deliver ? 1 : 0);
     return counted(c, cudaGetLastError());
 }

@@ -543,6 +543,28 @@ def test_randk_resnet18_shapes_layerwise_and_whole_vector():
             p.close()
 
 
+def _long_row_offsets():
+    # rows of more than 2^21 coordinates; the first 2^16 are 8192 blocks of 8 coordinates, each keeping one (most
+    # CTAs of the emit kernel then hold many blocks' first slots), then blocks of very different lengths
+    offs = list(range(0, 65536 + 1, 8))
+    for step in (100000, 31, 700001, 65536, 1234567, 5):
+        offs.append(offs[-1] + step)
+    return offs
+
+
+@pytest.mark.parametrize("n", [1, 3])
+def test_randk_long_rows_many_tiny_blocks_then_large_ones(n):
+    offs = _long_row_offsets()
+    d = offs[-1]
+    assert d >= 1 << 21
+    _pair_run(n, d, offs, RANDK, 0.01, _randn(n, d), steps=4)
+
+
+def test_randk_long_row_single_block_many_steps():
+    d = (1 << 21) + 4099
+    _pair_run(2, d, [0, d], RANDK, 0.02, _randn(2, d), steps=7, check_e_every=3)
+
+
 def test_randk_sets_follow_seed_and_iteration_count():
     n, d = 2, 50000
     gen = torch.Generator(device="cuda").manual_seed(3)

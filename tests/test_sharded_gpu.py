@@ -78,6 +78,12 @@ def test_shards_reproduce_the_whole_one_long_block(comp):
     _run(comp, 0.01, [0, d], 8, 2, steps=6, seed=3)
 
 
+def test_shards_reproduce_the_whole_randk_long_rows():
+    # long rows; a shard delivers nothing itself, the exchanged messages are scattered by compams_apply
+    d = (1 << 21) + 777
+    _run(RANDK, 0.01, [0, 300000, 300007, d], 4, 2, steps=3, seed=4)
+
+
 def test_sharded_run_matches_the_oracle():
     import oracle
     n_total, R, d = 4, 2, OFFS[-1]
