@@ -209,7 +209,7 @@ def config_entries():
     out.append(("C3/randk1%", lambda dev: _as_randk(W.config3(0.01, dev)), "randk", False))
     for lg in (20, 22, 24, 26, 27):
         for n in (1, 8, 32):
-            for mode in ("topk", "sign", "dense"):
+            for mode in ("topk", "sign", "dense") + (("randk",) if (lg, n) == (27, 32) else ()):
                 out.append(("C5/%s/d=2^%d/n=%d" % (mode, lg, n),
                             (lambda dev, lg=lg, n=n, mode=mode: W.sweep_point(1 << lg, n, mode, dev)), mode, False))
     return out
