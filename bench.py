@@ -107,7 +107,7 @@ def min_bytes(mode: str, n: int, d: int, bf16: bool = False) -> int:
 def algorithmic_bytes(kernel: str, n: int, d: int) -> int:
     """Bytes one launch of a dominant kernel must move: the sweeps read g and e and write x (12 B per
     worker-element, plus one sign bit for Block-Sign); the k = d kernel reads g and updates the state."""
-    return {"bs_sweep": 12 * n * d + n * d // 8, "topk_sweep": 12 * n * d, "dense_mean_amsgrad": (4 * n + 36) * d}[kernel]
+    return {"bs_sweep": 12 * n * d + n * d // 8, "topk_sweep": 12 * n * d, "dense_mean_amsgrad": (4 * n + 32) * d}[kernel]
 
 
 class ClockSampler:

@@ -131,7 +131,8 @@ int compams_create(compams_handle* out, int32_t n, int64_t d, const int64_t* blo
  *           Read only; must stay valid and unchanged until the enqueued work has run.
  *   theta   device; [d] fp32 parameters theta_t, overwritten with theta_{t+1}. 16-byte aligned.
  *
- * After the step: BUF_E holds e_{t+1}, BUF_GBAR holds gbar_t, BUF_M/V/VHAT the moments, and
+ * After the step: BUF_E holds e_{t+1}, BUF_GBAR holds gbar_t (while compams_record_average is on),
+ * BUF_M/V/VHAT the moments, and
  * the message buffers hold what each worker would have sent: for Top-k the k_b (index, value)
  * pairs of every (worker, block) - in no particular order inside a segment, ties at the
  * threshold magnitude resolved towards the lower index - and for Block-Sign one sign bit per
@@ -272,6 +273,16 @@ int compams_set_stream(compams_handle h, void* cuda_stream);
  * over the whole job (first_worker + local index on a sharded handle).
  */
 int compams_set_seed(compams_handle h, uint64_t seed, uint64_t iterations_done);
+
+/*
+ * compams_record_average - whether the server's update also stores the averaged compressed gradient gbar_t
+ * (Algorithm 2, the server's average), readable as COMPAMS_BUF_GBAR. gbar_t is an intermediate: theta, m, v and
+ * v-hat are computed from it in registers and nothing later reads it, so a new handle does not store it and the
+ * update moves 4 bytes per coordinate less. on != 0: stored from the next compams_step / compams_apply on;
+ * 0: not stored, and compams_get_buffer refuses COMPAMS_BUF_GBAR with INVALID_ARG. Every other result is
+ * bit-identical in both settings. A step captured in a CUDA graph keeps the setting it was captured with.
+ */
+int compams_record_average(compams_handle h, int on);
 
 /* compams_set_lr - learning rate eta_t for the following steps (Algorithm 2 allows it to vary
  * with t; Section 5.2 divides it by 10 at fixed epochs). */

@@ -93,6 +93,8 @@ def load_library() -> ctypes.CDLL:
     L.compams_set_stream.argtypes = [H, c.c_void_p]
     L.compams_set_seed.restype = c.c_int
     L.compams_set_seed.argtypes = [H, c.c_uint64, c.c_uint64]
+    L.compams_record_average.restype = c.c_int
+    L.compams_record_average.argtypes = [H, c.c_int]
     L.compams_set_lr.restype = c.c_int
     L.compams_set_lr.argtypes = [H, c.c_float]
     L.compams_get_state.restype = c.c_int
@@ -195,12 +197,14 @@ class CompAMS:
     def __init__(self, n: int, d: int, block_offsets: Sequence[int], compressor: int, k_ratio: float = 1.0,
                  lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
                  stream: Optional[torch.cuda.Stream] = None, n_total: Optional[int] = None, first_worker: int = 0,
-                 workspace: Optional[torch.Tensor] = None):
+                 workspace: Optional[torch.Tensor] = None, record_average: bool = False):
         """`n` workers live in this optimizer. With `n_total` > n they are workers `first_worker` ...
         `first_worker + n - 1` of a job whose other workers live in other optimizers (other GPUs): use
         compress() / apply() with an exchange of the message buffers in between instead of step().
         `workspace`: a contiguous CUDA uint8 tensor of at least workspace_bytes(...) bytes, 256-byte aligned,
-        that holds all of the optimizer's state (kept alive by this object); None: the library allocates."""
+        that holds all of the optimizer's state (kept alive by this object); None: the library allocates.
+        `record_average`: also store the averaged compressed gradient (buffer("gbar")); off, the update writes
+        4 bytes per coordinate less."""
         self._L = load_library()
         self.n, self.d = int(n), int(d)
         self.n_total = self.n if n_total is None else int(n_total)
@@ -223,6 +227,8 @@ class CompAMS:
             self._h = ctypes.c_void_p()
         _check(rc, "compams_create_sharded" if workspace is None else "compams_create_in_workspace")
         self.set_stream(stream if stream is not None else torch.cuda.current_stream())
+        if record_average:
+            self.record_average(True)
 
     # -- calls ---------------------------------------------------------------------------------
     def set_stream(self, stream: torch.cuda.Stream) -> None:
@@ -231,6 +237,10 @@ class CompAMS:
     def set_seed(self, seed: int, iterations_done: int = 0) -> None:
         """Random-k: the seed of the index sets and the number of iterations already done."""
         _check(self._L.compams_set_seed(self._h, int(seed), int(iterations_done)), "compams_set_seed")
+
+    def record_average(self, on: bool = True) -> None:
+        """Whether the following steps store the averaged compressed gradient, buffer("gbar")."""
+        _check(self._L.compams_record_average(self._h, 1 if on else 0), "compams_record_average")
 
     def set_lr(self, lr: float) -> None:
         _check(self._L.compams_set_lr(self._h, float(lr)), "compams_set_lr")

@@ -275,7 +275,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
             RC(dev_alloc(c, &t.bdirty, (size_t)t.nbucket));
         }
         t.status = c->status;
-        t.gbar = c->gbar;
+        t.gbar = nullptr;  // set by compams_record_average
         t.m = c->m;
         t.v = c->v;
         t.vhat = c->vhat;
@@ -301,7 +301,7 @@ int init_context(compams_context* c, const int64_t* block_offsets) {
         RC(dev_alloc(c, &c->scales[1], (size_t)c->n_total * (size_t)M));
         RC(dev_alloc(c, &s.tile_sum, (size_t)n * (size_t)c->tab.ntiles));
         RC(dev_alloc(c, &s.edge, (size_t)n * (size_t)c->tab.ntiles));
-        s.gbar = c->gbar;
+        s.gbar = nullptr;  // set by compams_record_average
         s.m = c->m;
         s.v = c->v;
         s.vhat = c->vhat;
@@ -592,6 +592,14 @@ int compams_set_seed(compams_handle c, uint64_t seed, uint64_t iterations_done) 
     return COMPAMS_OK;
 }
 
+int compams_record_average(compams_handle c, int on) {
+    if (!c) return COMPAMS_ERR_INVALID_ARG;
+    c->record_gbar = on != 0;
+    c->tk.gbar = c->record_gbar ? c->gbar : nullptr;
+    c->bs.gbar = c->record_gbar ? c->gbar : nullptr;
+    return COMPAMS_OK;
+}
+
 int compams_set_lr(compams_handle c, float lr) {
     if (!c || !(lr == lr)) return COMPAMS_ERR_INVALID_ARG;
     c->hp.lr = lr;
@@ -685,7 +693,9 @@ int compams_get_buffer(compams_handle c, int32_t which, void** dev_ptr, int64_t*
         case COMPAMS_BUF_M: p = c->m; cnt = c->d; break;
         case COMPAMS_BUF_V: p = c->v; cnt = c->d; break;
         case COMPAMS_BUF_VHAT: p = c->vhat; cnt = c->d; break;
-        case COMPAMS_BUF_GBAR: p = c->gbar; cnt = c->d; break;
+        case COMPAMS_BUF_GBAR:
+            if (!c->record_gbar) return COMPAMS_ERR_INVALID_ARG;  // not being written
+            p = c->gbar; cnt = c->d; break;
         case COMPAMS_BUF_TOPK_IDX: if (topk) { p = c->tk.idx; cnt = (int64_t)c->n_total * c->K; } break;
         case COMPAMS_BUF_TOPK_VAL: if (topk) { p = c->tk.val; cnt = (int64_t)c->n_total * c->K; } break;
         case COMPAMS_BUF_TOPK_SEG_OFFSETS: if (topk) { p = c->d_seg_off; cnt = c->M + 1; } break;

@@ -413,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
         amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);
         amsgrad_update(gb[2], mm.z, vv.z, hh.z, tt.z, hp);
         amsgrad_update(gb[3], mm.w, vv.w, hh.w, tt.w, hp);
-        store4(gbar + r, cls, make_float4(gb[0], gb[1], gb[2], gb[3]));
+        if (b.gbar) store4(gbar + r, cls, make_float4(gb[0], gb[1], gb[2], gb[3]));
         store4(m + r, cls, mm);
         store4(v + r, cls, vv);
         store4(vh + r, cls, hh);
@@ -424,7 +424,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
             if (r + k < len) {
                 float m1 = m[r + k], v1 = v[r + k], h1 = vh[r + k], t1 = th[r + k];
                 amsgrad_update(gb[k], m1, v1, h1, t1, hp);
-                gbar[r + k] = gb[k];
+                if (b.gbar) gbar[r + k] = gb[k];
                 m[r + k] = m1;
                 v[r + k] = v1;
                 vh[r + k] = h1;

@@ -122,6 +122,7 @@ struct compams_context {
     int32_t compressor = 0;
     double k_ratio = 1.0;
     bool identity = false;     // Top-k or Random-k with every k_b == d_b
+    bool record_gbar = false;  // the server kernels also write gbar_t (an intermediate; 4 bytes per coordinate and step)
     bool randk = false;        // Random-k: the kept sets are drawn, not selected
     uint64_t seed = 0;         // Random-k: seed of the index sets
     uint64_t iter = 0;         // iterations so far (Random-k keys its sets by the iteration index, from 1)

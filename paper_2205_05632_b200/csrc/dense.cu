@@ -2,7 +2,8 @@
 //
 // dense_mean_amsgrad: gbar = mean over workers of g_i (Algorithm 2, the server's average with C = identity,
 // so e stays 0), fused with the AMSGrad update (the moment, maximum and parameter updates). One pass over G [n, d] and the
-// four state vectors: (4n + 32) bytes per coordinate plus 4 for gbar.
+// four state vectors: (4n + 32) bytes per coordinate, plus 4 for gbar while the caller has asked for it to be recorded
+// (a null gbar: not written).
 //
 // amsgrad_bucket: the server update of the Top-k path. The scatter kernel has grouped the kept
 // (coordinate, value) entries of all workers by coordinate range; one CTA per range sums them in
@@ -46,7 +47,7 @@ __global__ void __launch_bounds__(kThreads, CTAS_PER_SM) dense_mean_amsgrad_kern
         amsgrad_update(gb.y, mm.y, vv.y, vh.y, th.y, hp);
         amsgrad_update(gb.z, mm.z, vv.z, vh.z, th.z, hp);
         amsgrad_update(gb.w, mm.w, vv.w, vh.w, th.w, hp);
-        *reinterpret_cast<float4*>(gbar + j) = gb;
+        if (gbar) *reinterpret_cast<float4*>(gbar + j) = gb;
         *reinterpret_cast<float4*>(m + j) = mm;
         *reinterpret_cast<float4*>(v + j) = vv;
         *reinterpret_cast<float4*>(vhat + j) = vh;
@@ -60,7 +61,7 @@ __global__ void __launch_bounds__(kThreads, CTAS_PER_SM) dense_mean_amsgrad_kern
         float gb = mean_from_acc(a, hp);
         float mm = m[j], vv = v[j], vh = vhat[j], th = theta[j];
         amsgrad_update(gb, mm, vv, vh, th, hp);
-        gbar[j] = gb;
+        if (gbar) gbar[j] = gb;
         m[j] = mm;
         v[j] = vv;
         vhat[j] = vh;
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
         amsgrad_update(gb.y, mm.y, vv.y, vh.y, th.y, hp);
         amsgrad_update(gb.z, mm.z, vv.z, vh.z, th.z, hp);
         amsgrad_update(gb.w, mm.w, vv.w, vh.w, th.w, hp);
-        *reinterpret_cast<float4*>(b.gbar + j) = gb;
+        if (b.gbar) *reinterpret_cast<float4*>(b.gbar + j) = gb;
         *reinterpret_cast<float4*>(b.m + j) = mm;
         *reinterpret_cast<float4*>(b.v + j) = vv;
         *reinterpret_cast<float4*>(b.vhat + j) = vh;
@@ -149,7 +150,7 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
             const float gb = mean_from_acc(ak, hp);
             float m1 = b.m[j + k], v1 = b.v[j + k], h1 = b.vhat[j + k], t1 = theta[j + k];
             amsgrad_update(gb, m1, v1, h1, t1, hp);
-            b.gbar[j + k] = gb;
+            if (b.gbar) b.gbar[j + k] = gb;
             b.m[j + k] = m1;
             b.v[j + k] = v1;
             b.vhat[j + k] = h1;
@@ -163,21 +164,22 @@ cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, flo
     int grid = (int)((groups + kThreads - 1) / kThreads);
     if (grid < 1) grid = 1;
     const bool many_rows = c->n >= 6;
+    float* gbar = c->record_gbar ? c->gbar : nullptr;
     if (c->grad_bf16) {
         const bf16_bits* g = (const bf16_bits*)grads;
         if (many_rows)
-            dense_mean_amsgrad_kernel<bf16_bits, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+            dense_mean_amsgrad_kernel<bf16_bits, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
                                                                                       c->vhat, theta, c->hp);
         else
-            dense_mean_amsgrad_kernel<bf16_bits, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+            dense_mean_amsgrad_kernel<bf16_bits, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
                                                                                       c->vhat, theta, c->hp);
     } else {
         const float* g = (const float*)grads;
         if (many_rows)
-            dense_mean_amsgrad_kernel<float, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+            dense_mean_amsgrad_kernel<float, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
                                                                                   c->vhat, theta, c->hp);
         else
-            dense_mean_amsgrad_kernel<float, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, c->gbar, c->m, c->v,
+            dense_mean_amsgrad_kernel<float, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
                                                                                   c->vhat, theta, c->hp);
     }
     return counted(c, cudaGetLastError());

@@ -64,7 +64,7 @@ class Pair:
         self.offsets = np.asarray(block_offsets, dtype=np.int64)
         self.compressor = compressor
         hp = dict(lr=lr, beta1=beta1, beta2=beta2, eps=eps)
-        self.gpu = CompAMS(n, d, self.offsets, compressor, k_ratio, **hp)
+        self.gpu = CompAMS(n, d, self.offsets, compressor, k_ratio, record_average=True, **hp)
         self.cpu = oracle.Oracle(n, d, self.offsets, compressor, k_ratio, **hp)
         sizes = np.diff(self.offsets)
         if seed is not None:  # Random-k: the same seed for the index sets on both sides

@@ -20,7 +20,7 @@ def test_two_captured_steps_replay_like_eager_steps(comp, ratio):
     offs = [0, 3000, 40000, d]
     gen = torch.Generator(device="cuda").manual_seed(6)
     G = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(9)]
-    eager = CompAMS(n, d, offs, comp, ratio)
+    eager = CompAMS(n, d, offs, comp, ratio, record_average=True)
     theta_eager = torch.zeros(d, device="cuda")
     for g in G:
         eager.step(g, theta_eager)
@@ -30,7 +30,7 @@ def test_two_captured_steps_replay_like_eager_steps(comp, ratio):
     theta = torch.zeros(d, device="cuda")
     slots = [torch.empty(n, d, device="cuda") for _ in range(2)]
     with torch.cuda.stream(side):
-        opt = CompAMS(n, d, offs, comp, ratio, stream=side)
+        opt = CompAMS(n, d, offs, comp, ratio, stream=side, record_average=True)
         opt.step(G[0].clone(), theta)          # warm-up: from here on the host-side switches alternate
         side.synchronize()
         graph = torch.cuda.CUDAGraph()

@@ -111,8 +111,8 @@ def test_gradient_buffer_off_the_16_byte_grid(shift):
     n, d = 3, 2 * 8192 + 4101
     offs = [0, 4099, d]
     for comp, ratio in ((TOPK, 0.05), (BLOCKSIGN, 1.0), (TOPK, 1.0)):
-        a = CompAMS(n, d, offs, comp, ratio)
-        b = CompAMS(n, d, offs, comp, ratio)
+        a = CompAMS(n, d, offs, comp, ratio, record_average=True)
+        b = CompAMS(n, d, offs, comp, ratio, record_average=True)
         ta = torch.zeros(d, device="cuda")
         tb = torch.zeros(d, device="cuda")
         gen = torch.Generator(device="cuda").manual_seed(77)
@@ -445,6 +445,37 @@ def test_learning_rate_schedule_matches_the_oracle(comp, ratio):
         p.close()
 
 
+@pytest.mark.parametrize("comp,ratio", [(TOPK, 0.01), (TOPK, 1.0), (BLOCKSIGN, 1.0), (RANDK, 0.02)])
+def test_the_average_is_stored_only_on_request_and_changes_nothing_else(comp, ratio):
+    # gbar_t is an intermediate of the server's update: a new handle does not store it, asking for it is refused,
+    # and every result of the step is the same bits with and without it
+    n, d = 3, 5 * 8192 + 77   # the last bucket and the last float4 group are partial
+    offs = [0, 4099, 30001, d]
+    gen = torch.Generator(device="cuda").manual_seed(8)
+    G = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(4)]
+    plain, rec = CompAMS(n, d, offs, comp, ratio), CompAMS(n, d, offs, comp, ratio, record_average=True)
+    tp, tr = torch.zeros(d, device="cuda"), torch.zeros(d, device="cuda")
+    for t, g in enumerate(G):
+        plain.step(g, tp)
+        rec.step(g, tr)
+        if t == 1:
+            with pytest.raises(CompAMSError):
+                plain.buffer("gbar")
+            rec.buffer("gbar")
+    assert torch.equal(tp.view(torch.int32), tr.view(torch.int32))
+    for name in ("E", "m", "v", "vhat"):
+        assert torch.equal(plain.buffer(name).view(torch.int32), rec.buffer(name).view(torch.int32)), name
+    # switched on later, the next step stores it; it equals the recorded handle's
+    plain.record_average(True)
+    g = torch.randn(n, d, generator=gen, device="cuda")
+    plain.step(g, tp)
+    rec.step(g, tr)
+    assert torch.equal(plain.buffer("gbar").view(torch.int32), rec.buffer("gbar").view(torch.int32))
+    assert plain.check_status() == 0 and rec.check_status() == 0
+    plain.close()
+    rec.close()
+
+
 def test_calls_out_of_order_are_rejected():
     # compress opens an iteration and apply closes it: in between the residual is not final, so the
     # state cannot be read or replaced, and neither call may come twice in a row
@@ -460,7 +491,7 @@ def test_calls_out_of_order_are_rejected():
                      lambda: opt.get_state(), lambda: opt.set_state({"m": torch.zeros(d, device="cuda")})):
             with pytest.raises(CompAMSError):
                 call()
-        opt.buffer("gbar")                    # buffers that the open iteration does not touch stay readable
+        opt.buffer("m")                       # buffers that the open iteration does not touch stay readable
         opt.apply(theta)
         opt.step(G, theta)                    # and the handle goes on as usual
         assert opt.check_status() == 0
@@ -598,7 +629,7 @@ def test_steps_on_a_side_stream_match_the_default_stream(comp, ratio):
     offs = [0, 3000, 30000, d]
     gen = torch.Generator(device="cuda").manual_seed(12)
     G = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(5)]
-    ref = CompAMS(n, d, offs, comp, ratio)
+    ref = CompAMS(n, d, offs, comp, ratio, record_average=True)
     theta_ref = torch.zeros(d, device="cuda")
     for g in G:
         ref.step(g, theta_ref)
@@ -606,7 +637,7 @@ def test_steps_on_a_side_stream_match_the_default_stream(comp, ratio):
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     theta = torch.zeros(d, device="cuda")
     with torch.cuda.stream(s1):
-        opt = CompAMS(n, d, offs, comp, ratio, stream=s1)
+        opt = CompAMS(n, d, offs, comp, ratio, stream=s1, record_average=True)
         for g in G[:3]:
             staged = g.clone()          # produced on s1, consumed by the step on s1
             opt.step(staged, theta)

@@ -28,9 +28,10 @@ def _swap_rows(shards):
 def _run(comp, ratio, offs, n_total, R, steps=5, seed=0):
     d = offs[-1]
     gen = torch.Generator(device="cuda").manual_seed(seed)
-    whole = CompAMS(n_total, d, offs, comp, ratio)
+    whole = CompAMS(n_total, d, offs, comp, ratio, record_average=True)
     per = n_total // R
-    shards = [CompAMS(per, d, offs, comp, ratio, n_total=n_total, first_worker=r * per) for r in range(R)]
+    shards = [CompAMS(per, d, offs, comp, ratio, n_total=n_total, first_worker=r * per, record_average=True)
+              for r in range(R)]
     theta = 0.1 * torch.randn(d, generator=gen, device="cuda")
     thetas = [theta.clone() for _ in range(R)]
     for t in range(steps):

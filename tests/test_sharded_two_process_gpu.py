@@ -52,6 +52,7 @@ def _rank(rank, world, port, comp, ratio, steps):
         w.n = n_total = world * n_local
         theta = w.start()
         opt = ShardedCompAMS(n_local, w.d, w.block_offsets, comp, ratio)
+        opt.opt.record_average(True)
         ref = oracle.Oracle(n_total, w.d, w.block_offsets, comp, ratio)
         if comp == 2:
             opt.opt.set_seed(11)

@@ -43,8 +43,8 @@ def test_handle_in_caller_memory_matches_the_self_allocating_handle(comp, ratio)
     need = workspace_bytes(n, d, offs, comp, ratio)
     ws = torch.full((need,), 0xA5, dtype=torch.uint8, device="cuda")  # garbage: the handle must initialise its state
     assert ws.data_ptr() % 256 == 0
-    a = CompAMS(n, d, offs, comp, ratio, workspace=ws)
-    b = CompAMS(n, d, offs, comp, ratio)
+    a = CompAMS(n, d, offs, comp, ratio, workspace=ws, record_average=True)
+    b = CompAMS(n, d, offs, comp, ratio, record_average=True)
     gen = torch.Generator(device="cuda").manual_seed(4)
     ta, tb = torch.zeros(d, device="cuda"), torch.zeros(d, device="cuda")
     for _ in range(4):
