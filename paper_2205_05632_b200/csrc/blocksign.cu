@@ -305,7 +305,7 @@ __device__ __forceinline__ void transpose32x4(uint32_t (&x)[4], int lane) {
 // round. The kernel is bound by instruction issue: the fixed cost of the transposition (36 shuffles per round)
 // pays from about two dozen workers up (n = 32, d = 2^27: step 9.23 -> 8.87 ms; n = 16: no change; n = 8: 3 %
 // slower, hence the two forms).
-template <bool TABLES>
+template <bool TABLES, bool RECORD>
 __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffers b, float* __restrict__ theta,
                                                                HyperParams hp,
                                                                const __grid_constant__ SegParams sp_) {
@@ -413,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
         amsgrad_update(gb[1], mm.y, vv.y, hh.y, tt.y, hp);
         amsgrad_update(gb[2], mm.z, vv.z, hh.z, tt.z, hp);
         amsgrad_update(gb[3], mm.w, vv.w, hh.w, tt.w, hp);
-        if (b.gbar) store4(gbar + r, cls, make_float4(gb[0], gb[1], gb[2], gb[3]));
+        if constexpr (RECORD) store4(gbar + r, cls, make_float4(gb[0], gb[1], gb[2], gb[3]));
         store4(m + r, cls, mm);
         store4(v + r, cls, vv);
         store4(vh + r, cls, hh);
@@ -424,7 +424,7 @@ __global__ void __launch_bounds__(kThreads, 5) bs_apply_kernel(Tables t, BsBuffe
             if (r + k < len) {
                 float m1 = m[r + k], v1 = v[r + k], h1 = vh[r + k], t1 = th[r + k];
                 amsgrad_update(gb[k], m1, v1, h1, t1, hp);
-                if (b.gbar) gbar[r + k] = gb[k];
+                if constexpr (RECORD) gbar[r + k] = gb[k];
                 m[r + k] = m1;
                 v[r + k] = v1;
                 vh[r + k] = h1;
@@ -475,15 +475,15 @@ cudaError_t launch_bs_apply(compams_context* c, float* theta) {
     t.n = c->n_total;  // the average runs over every worker's message
     const dim3 grid((unsigned)c->tab.ntiles * kWarps);
     const bool tables = c->n_total >= kApplyTablesFrom;
-    if (c->n == c->n_total)
-        return counted(c, tables ? launch_after(bs_apply_kernel<true>, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp)
-                                 : launch_after(bs_apply_kernel<false>, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp));
+    // four builds: the inner sum by tables or worker by worker; gbar stored or not (a run-time branch around the
+    // store slowed the kernel by a tenth)
+    void (*kernel)(Tables, BsBuffers, float*, HyperParams, const SegParams) =
+        tables ? (b.gbar ? bs_apply_kernel<true, true> : bs_apply_kernel<true, false>)
+               : (b.gbar ? bs_apply_kernel<false, true> : bs_apply_kernel<false, false>);
+    if (c->n == c->n_total) return counted(c, launch_after(kernel, grid, dim3(kThreads), c->stream, t, b, theta, c->hp, c->segp));
     // sharded workers: the other workers' messages were written by the caller's exchange, which is
     // ordered on the stream like any kernel; a plain launch waits for it
-    if (tables)
-        bs_apply_kernel<true><<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
-    else
-        bs_apply_kernel<false><<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
+    kernel<<<grid, dim3(kThreads), 0, c->stream>>>(t, b, theta, c->hp, c->segp);
     return counted(c, cudaGetLastError());
 }
 

@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(kThreads, CTAS_PER_SM) dense_mean_amsgrad_kern
 // run to run in the last bit of gbar, which stays inside the tolerance the step is specified to. Entries
 // that did not fit their bucket were added to acc[] by the scatter kernel and are folded in (and acc
 // cleared) here.
+template <bool RECORD>
 __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, TopkBuffers b, float* __restrict__ theta,
                                                                      HyperParams hp) {
     static_assert(kBucketSpan == 4 * kThreads, "one float4 group per thread");
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
         amsgrad_update(gb.y, mm.y, vv.y, vh.y, th.y, hp);
         amsgrad_update(gb.z, mm.z, vv.z, vh.z, th.z, hp);
         amsgrad_update(gb.w, mm.w, vv.w, vh.w, th.w, hp);
-        if (b.gbar) *reinterpret_cast<float4*>(b.gbar + j) = gb;
+        if constexpr (RECORD) *reinterpret_cast<float4*>(b.gbar + j) = gb;
         *reinterpret_cast<float4*>(b.m + j) = mm;
         *reinterpret_cast<float4*>(b.v + j) = vv;
         *reinterpret_cast<float4*>(b.vhat + j) = vh;
@@ -150,7 +151,7 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
             const float gb = mean_from_acc(ak, hp);
             float m1 = b.m[j + k], v1 = b.v[j + k], h1 = b.vhat[j + k], t1 = theta[j + k];
             amsgrad_update(gb, m1, v1, h1, t1, hp);
-            if (b.gbar) b.gbar[j + k] = gb;
+            if constexpr (RECORD) b.gbar[j + k] = gb;
             b.m[j + k] = m1;
             b.v[j + k] = v1;
             b.vhat[j + k] = h1;
@@ -159,35 +160,30 @@ __global__ void __launch_bounds__(kThreads, 5) amsgrad_bucket_kernel(int64_t d, 
     }
 }
 
+// gbar stored or not: a null pointer here (as a template parameter this kernel ran 4 % slower), a template
+// parameter in amsgrad_bucket and bs_apply (where the run-time branch around the store cost up to a tenth).
+template <typename GT>
+static void launch_dense_typed(compams_context* c, const GT* g, float* theta, int grid) {
+    float* gbar = c->record_gbar ? c->gbar : nullptr;
+    if (c->n >= 6)
+        dense_mean_amsgrad_kernel<GT, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v, c->vhat, theta, c->hp);
+    else
+        dense_mean_amsgrad_kernel<GT, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v, c->vhat, theta, c->hp);
+}
+
 cudaError_t launch_dense_mean_amsgrad(compams_context* c, const void* grads, float* theta) {
     int64_t groups = c->d >> 2;
     int grid = (int)((groups + kThreads - 1) / kThreads);
     if (grid < 1) grid = 1;
-    const bool many_rows = c->n >= 6;
-    float* gbar = c->record_gbar ? c->gbar : nullptr;
-    if (c->grad_bf16) {
-        const bf16_bits* g = (const bf16_bits*)grads;
-        if (many_rows)
-            dense_mean_amsgrad_kernel<bf16_bits, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
-                                                                                      c->vhat, theta, c->hp);
-        else
-            dense_mean_amsgrad_kernel<bf16_bits, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
-                                                                                      c->vhat, theta, c->hp);
-    } else {
-        const float* g = (const float*)grads;
-        if (many_rows)
-            dense_mean_amsgrad_kernel<float, 8><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
-                                                                                  c->vhat, theta, c->hp);
-        else
-            dense_mean_amsgrad_kernel<float, 6><<<grid, kThreads, 0, c->stream>>>(c->n, c->d, g, gbar, c->m, c->v,
-                                                                                  c->vhat, theta, c->hp);
-    }
+    if (c->grad_bf16) launch_dense_typed(c, (const bf16_bits*)grads, theta, grid);
+    else launch_dense_typed(c, (const float*)grads, theta, grid);
     return counted(c, cudaGetLastError());
 }
 
 cudaError_t launch_amsgrad(compams_context* c, float* theta) {
-    return counted(c, launch_after(amsgrad_bucket_kernel, dim3((unsigned)c->tk.nbucket), dim3(kThreads), c->stream, c->d, c->tk, theta,
-                        c->hp));
+    const dim3 grid((unsigned)c->tk.nbucket);
+    return counted(c, c->tk.gbar ? launch_after(amsgrad_bucket_kernel<true>, grid, dim3(kThreads), c->stream, c->d, c->tk, theta, c->hp)
+                                 : launch_after(amsgrad_bucket_kernel<false>, grid, dim3(kThreads), c->stream, c->d, c->tk, theta, c->hp));
 }
 
 }  // namespace compams
