@@ -163,6 +163,9 @@ int build_tiles(compams_context* c, const std::vector<int32_t>& blocks, bool top
             if (segs[s].cap == 0) continue;  // never predicts: always the dense passes, no select needed
             (segs[s].cap <= single_max ? small_l : big_l).push_back((int32_t)s);
         }
+        // one-CTA lists are worked on longest first (their CTAs differ in length by the lists' lengths)
+        std::stable_sort(small_l.begin(), small_l.end(),
+                         [&](int32_t a, int32_t b) { return segs[(size_t)a].cap > segs[(size_t)b].cap; });
         RC(dev_upload(c, &c->sel_small, small_l));
         RC(dev_upload(c, &c->sel_big, big_l));
         c->n_sel_small = (int)small_l.size();

@@ -369,8 +369,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     __shared__ uint32_t scratch[kSelWarps];
     __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt;
     const int lane = threadIdx.x & 31;
-    const int i = (int)(blockIdx.x / (unsigned)nlist);
-    const int seg = seg_list[blockIdx.x % (unsigned)nlist];
+    // the lists come longest first, every worker's copy of one block side by side: the CTAs that take longest
+    // start first and the last wave holds the shortest lists
+    const int i = (int)(blockIdx.x % (unsigned)t.n);
+    const int seg = seg_list[blockIdx.x / (unsigned)t.n];
     const size_t sg = (size_t)i * t.nseg + seg;
     const SegInfo* si = t.segs + seg;
     SegState* st = b.seg + sg;
