@@ -301,9 +301,12 @@ __device__ __forceinline__ void margin_held(SegState* st) {
 }
 
 constexpr int kSelUnroll = 4;   // candidate loads in flight per thread while scanning a list
-constexpr int kSelThreads = 1024;  // many threads per list keep enough loads in flight; two such CTAs share an SM
-                                   // (32 registers): layer-wise selection on ResNet-50 shapes 0.212 -> 0.180 ms
-constexpr int kSelWarps = kSelThreads / 32;
+// One CTA per short list, 2048 threads to the SM at 32 registers. 1024 threads per list keep enough loads in flight
+// to finish one list soonest (few lists: d = 2^20, n = 8: step 0.051 ms against 0.058 with 512); with more lists
+// than the GPU holds CTAs, 512 threads per list and twice as many lists in flight get through them sooner
+// (ResNet-50 shapes layer-wise, n = 32, 1696 lists: select 0.121 -> 0.111 ms; with 256: 0.178).
+constexpr int kSelThreads = 1024;
+constexpr int kSelThreadsMany = 512;
 
 // Adds the `pred` lanes of a warp to a shared counter with one atomic; returns this lane's slot.
 __device__ __forceinline__ uint32_t warp_slot(bool pred, uint32_t* counter, int lane) {
@@ -322,7 +325,7 @@ __device__ __forceinline__ uint32_t warp_slot(bool pred, uint32_t* counter, int 
 struct BinScan {
     uint32_t incl, excl;
 };
-template <int NT = kSelThreads>
+template <int NT>
 __device__ __forceinline__ BinScan scan_from_top(const uint32_t* hm, int nb, uint32_t* scratch, uint32_t* total) {
     const int per = nb / NT > 0 ? nb / NT : 1;
     uint32_t sum = 0;
@@ -337,7 +340,7 @@ __device__ __forceinline__ BinScan scan_from_top(const uint32_t* hm, int nb, uin
 }
 // The thread whose bins hold the `target`-th entry from the top writes
 // sh_out[0] = bin, sh_out[1] = entries above the bin, sh_out[2] = entries in the bin.
-template <int NT = kSelThreads>
+template <int NT>
 __device__ __forceinline__ void locate(const uint32_t* hm, int nb, const BinScan& sc, uint32_t target, uint32_t* sh_out) {
     if (sc.excl < target && target <= sc.incl) {
         const int per = nb / NT > 0 ? nb / NT : 1;
@@ -360,13 +363,14 @@ __device__ __forceinline__ uint32_t offset_digit(uint32_t xbits, uint32_t tau_ha
     return dg < (uint32_t)(kSelBins - 1) ? dg : (uint32_t)(kSelBins - 1);
 }
 
-__global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
+template <int NT>
+__global__ void __launch_bounds__(NT, 2048 / NT) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                int nlist) {
     dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint32_t local[kSelBins];  // histogram of the list
     __shared__ uint2 surv[kSurvCap];
-    __shared__ uint32_t scratch[kSelWarps];
+    __shared__ uint32_t scratch[NT / 32];
     __shared__ uint32_t sh_bin[3], sh_edge[3], sh_base, sh_wcnt, sh_scnt;
     const int lane = threadIdx.x & 31;
     // the lists come longest first, every worker's copy of one block side by side: the CTAs that take longest
@@ -394,14 +398,14 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     auto digit0 = [&](uint32_t xbits) -> uint32_t { return offset_digit(xbits, tau_hat, S); };
 
     // ---- pass 0: histogram of the key offsets above tau_hat in bins of 2^S; the last bin is open-ended
-    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads) local[k] = 0u;
+    for (int k = threadIdx.x; k < kSelBins; k += NT) local[k] = 0u;
     if (threadIdx.x == 0) sh_scnt = 0u;
     __syncthreads();
-    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kSelThreads) {
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * NT) {
         uint32_t y[kSelUnroll];
 #pragma unroll
         for (int u = 0; u < kSelUnroll; ++u) {
-            const uint32_t p = p0 + u * kSelThreads + threadIdx.x;
+            const uint32_t p = p0 + u * NT + threadIdx.x;
             y[u] = p < hi ? list[p].y : 0xffffffffu;  // no candidate has this pattern (NaN)
         }
 #pragma unroll
@@ -418,12 +422,12 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     __syncthreads();
     uint32_t total;
     {
-        const BinScan sc = scan_from_top(local, kSelBins, scratch, &total);
+        const BinScan sc = scan_from_top<NT>(local, kSelBins, scratch, &total);
         const uint32_t want = want_candidates(kb, st->boost);
         if (threadIdx.x == 0) sh_edge[0] = 0xffffffffu;  // "fewer than `want` candidates"
         __syncthreads();
-        locate(local, kSelBins, sc, kb, sh_bin);
-        locate(local, kSelBins, sc, want, sh_edge);
+        locate<NT>(local, kSelBins, sc, kb, sh_bin);
+        locate<NT>(local, kSelBins, sc, want, sh_edge);
     }
     __syncthreads();
     const uint32_t b0 = sh_bin[0];
@@ -433,10 +437,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
     const bool take_all0 = (c0 == k_rem);
     // the number of winners, from the histogram
     uint32_t mine = 0;
-    for (int k = threadIdx.x; k < kSelBins; k += kSelThreads)
+    for (int k = threadIdx.x; k < kSelBins; k += NT)
         if ((uint32_t)k > b0 || (take_all0 && (uint32_t)k == b0)) mine += local[k];
     uint32_t my_winners;
-    block_inclusive_scan<kSelWarps>(mine, scratch, &my_winners);
+    block_inclusive_scan<NT / 32>(mine, scratch, &my_winners);
     __syncthreads();
     if (b0 == (uint32_t)(kSelBins - 1) && !take_all0) {
         // the threshold lies in the open-ended bin: the prediction was far off, let the dense passes decide
@@ -457,11 +461,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
         sh_wcnt = 0u;
     }
     __syncthreads();
-    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * kSelThreads) {
+    for (uint32_t p0 = lo; p0 < hi; p0 += kSelUnroll * NT) {
         uint2 cvs[kSelUnroll];
 #pragma unroll
         for (int u = 0; u < kSelUnroll; ++u) {
-            const uint32_t p = p0 + u * kSelThreads + threadIdx.x;
+            const uint32_t p = p0 + u * NT + threadIdx.x;
             cvs[u] = p < hi ? list[p] : make_uint2(0u, 0xffffffffu);
         }
 #pragma unroll
@@ -513,7 +517,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
             const uint32_t o = (cv.y & 0x7fffffffu) - tau_hat;
             return ((unsigned long long)(o & lowmask) << 32) | (unsigned long long)(0xffffffffu - cv.x);
         };
-        for (uint32_t q0 = 0; q0 < nsurv; q0 += kSelThreads) {  // uniform trip count: the loop holds barriers
+        for (uint32_t q0 = 0; q0 < nsurv; q0 += NT) {  // uniform trip count: the loop holds barriers
             const uint32_t q = q0 + threadIdx.x;
             bool kept = false;
             uint2 cv = make_uint2(0u, 0u);
@@ -526,7 +530,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) topk_select_kernel(Tables t, T
                 if (beaten == k_rem - 1u) sh_edge[1] = (cv.y & 0x7fffffffu);  // the k-th largest key overall
             }
             uint32_t tot3;
-            const uint32_t incl = block_inclusive_scan<kSelWarps>(kept ? 1u : 0u, scratch, &tot3);
+            const uint32_t incl = block_inclusive_scan<NT / 32>(kept ? 1u : 0u, scratch, &tot3);
             if (threadIdx.x == 0) sh_base = tot3 ? atomicAdd(&st->emit_count, tot3) : 0u;
             __syncthreads();
             if (kept) {
@@ -1373,9 +1377,15 @@ static cudaError_t launch_chained(compams_context* c, void (*kernel)(KArgs...), 
 cudaError_t launch_topk_select(compams_context* c) {
     cudaError_t e = cudaSuccess;
     const TopkBuffers b = own_rows(c);
-    if (c->n_sel_small > 0)
-        e = launch_chained(c, topk_select_kernel, dim3((unsigned)((int64_t)c->n * c->n_sel_small)), dim3(kSelThreads),
-                           c->tab, b, (const int32_t*)c->sel_small, c->n_sel_small);
+    if (c->n_sel_small > 0) {
+        const int64_t lists = (int64_t)c->n * c->n_sel_small;
+        if (lists >= 4 * (int64_t)c->num_sms)
+            e = launch_chained(c, topk_select_kernel<kSelThreadsMany>, dim3((unsigned)lists), dim3(kSelThreadsMany), c->tab, b,
+                               (const int32_t*)c->sel_small, c->n_sel_small);
+        else
+            e = launch_chained(c, topk_select_kernel<kSelThreads>, dim3((unsigned)lists), dim3(kSelThreads), c->tab, b,
+                               (const int32_t*)c->sel_small, c->n_sel_small);
+    }
     if (e != cudaSuccess || c->n_sel_big == 0) return e;
     const dim3 grid((unsigned)((int64_t)c->n * c->n_sel_big * c->sel_parts));
     e = launch_chained(c, topk_selhist_kernel, grid, dim3(kThreads), c->tab, b, (const int32_t*)c->sel_big, c->n_sel_big,
