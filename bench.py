@@ -184,7 +184,7 @@ def workload_config(pt):
     n, d = pt["n"], 1 << pt["log2d"]
     return {
         "workload": describe(pt), "n_workers": n, "d": d, "compressor": "topk", "k_ratio": 0.01,
-        "l2": "inputs larger than L2 (each [n,d] buffer is %.1f GB; ring of 2 gradient batches)" % (n * d * 4 / 1e9),
+        "l2": "inputs larger than L2 (each [n,d] buffer is %.1f GB)" % (n * d * 4 / 1e9),
         "parallelism": "replicas only",
     }
 
@@ -215,26 +215,63 @@ def config_entries():
     return out
 
 
+FEED_RING = 8                 # gradient batches kept when they fit the budget below
+FEED_RING_BYTES = 48 << 30
+FEED_SHIFT = 64               # elements between the windows of consecutive steps: whole 128-byte lines in fp32 and bf16
+FEED_PERIOD = 509             # windows before the offsets repeat
+
+
+class GradientFeed:
+    """A different gradient batch for every step, with nothing generated inside the timed region. Under error
+    feedback a short cycle of batches is not a stand-in for training: with two alternating batches the
+    accumulators settle into a period-two pattern whose selection threshold swings from step to step, which fresh
+    gradients never do. So: a ring of FEED_RING batches drawn in advance when that fits FEED_RING_BYTES; for
+    larger one-block workloads of independent N(0,1) entries one buffer of n d + tail draws, of which step t takes
+    the window at offset FEED_SHIFT (t mod FEED_PERIOD) viewed as [n, d] - every coordinate sees an independent
+    draw each step, and the rows keep their alignment; otherwise (no such workload exists among the entries) a
+    ring of as many batches as fit, at least two."""
+
+    def __init__(self, w, bf16=False):
+        per = w.n * w.d * 4
+        self.n, self.d, self.flat, self.ring = w.n, w.d, None, None
+        if FEED_RING * per <= FEED_RING_BYTES or not W.iid_normal(w):
+            count = max(2, min(FEED_RING, FEED_RING_BYTES // per))
+            self.ring = [w.grads() for _ in range(count)]
+            if bf16:
+                self.ring = [g.bfloat16() for g in self.ring]
+            self.kind = "ring of %d gradient batches" % count
+        else:
+            self.flat = W.grads_with_tail(w, FEED_SHIFT * (FEED_PERIOD - 1))
+            if bf16:
+                self.flat = self.flat.bfloat16()
+            self.kind = "a window moving by %d elements per step over one buffer of n d + %d draws" % (
+                FEED_SHIFT, FEED_SHIFT * (FEED_PERIOD - 1))
+
+    def __call__(self, t):
+        if self.ring is not None:
+            return self.ring[t % len(self.ring)]
+        o = FEED_SHIFT * (t % FEED_PERIOD)
+        return self.flat[o:o + self.n * self.d].view(self.n, self.d)
+
+
 def time_entry(name, build, mode, bf16, steps, warmup, peak, peak_kind, cache):
     """Creates the workload and its optimizer, runs `warmup` + `steps` steps and returns the entry's record."""
     from paper_2205_05632_b200 import CompAMS
     w = build("cuda")
     key = (w.n, w.d, name.split("/")[0], bf16)
     if key in cache:  # the modes of one sweep point consume the same gradients
-        theta0, ring = cache[key]
+        theta0, feed = cache[key]
     else:
         cache.clear()
         torch.cuda.empty_cache()
         theta0 = w.start()
-        ring = [w.grads(), w.grads()]
-        if bf16:
-            ring = [g.bfloat16() for g in ring]
-        cache[key] = (theta0, ring)
+        feed = GradientFeed(w, bf16)
+        cache[key] = (theta0, feed)
     theta = theta0.clone()
     opt = CompAMS(w.n, w.d, w.block_offsets, w.compressor, w.k_ratio, w.lr, w.beta1, w.beta2, w.eps)
     try:
         for t in range(warmup):
-            opt.step(ring[t % 2], theta)
+            opt.step(feed(t), theta)
         opt.check_status()
         st0 = opt.buffer("status").cpu().tolist()
         l0 = opt.launch_count()
@@ -242,7 +279,7 @@ def time_entry(name, build, mode, bf16, steps, warmup, peak, peak_kind, cache):
         torch.cuda.synchronize()
         s.record()
         for t in range(steps):
-            opt.step(ring[(warmup + t) % 2], theta)
+            opt.step(feed(warmup + t), theta)
         e.record()
         torch.cuda.synchronize()
         opt.check_status()
@@ -256,8 +293,8 @@ def time_entry(name, build, mode, bf16, steps, warmup, peak, peak_kind, cache):
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
                 opt.set_stream(torch.cuda.current_stream())
-                opt.step(ring[0], theta)
-                opt.step(ring[1], theta)
+                opt.step(feed(0), theta)
+                opt.step(feed(1), theta)
             opt.set_stream(torch.cuda.current_stream())
             pairs = max(steps // 2, 1)
             graph.replay()
@@ -276,7 +313,8 @@ def time_entry(name, build, mode, bf16, steps, warmup, peak, peak_kind, cache):
     gbs = mb / ms / 1e6
     fits_l2 = 2 * w.n * w.d * 4 <= L2_BYTES
     rec = {"name": name, "mode": mode, "n": w.n, "d": w.d, "blocks": int(len(w.block_offsets) - 1),
-           "ms": ms, "elems_per_s": w.n * w.d / ms * 1e3, "min_bytes": mb, "launches_per_step": launches}
+           "ms": ms, "elems_per_s": w.n * w.d / ms * 1e3, "min_bytes": mb, "launches_per_step": launches,
+           "gradients": feed.kind}
     if fits_l2:
         rec["note"] = "launch-bound: inputs fit L2, no HBM fraction"
         rec["ms_as_cuda_graph"] = graph_ms
@@ -369,7 +407,7 @@ def main():
     ap.add_argument("--no-headline", action="store_true", help="time only the entries selected with --only")
     ap.add_argument("--only", nargs="*", default=None, help="names (or prefixes) of the 'configs' entries to time")
     ap.add_argument("--config-steps", type=int, default=20)
-    ap.add_argument("--config-warmup", type=int, default=8)
+    ap.add_argument("--config-warmup", type=int, default=40)
     ap.add_argument("--e2e-steps", type=int, default=3)
     args = ap.parse_args()
 
@@ -394,12 +432,12 @@ def main():
         n, d = pt["n"], 1 << pt["log2d"]
         w = W.sweep_point(d, n, "topk", device)
         theta = w.start()
-        ring = [w.grads(), w.grads()]
+        feed = GradientFeed(w)
         opt = CompAMS(w.n, w.d, w.block_offsets, w.compressor, w.k_ratio, w.lr, w.beta1, w.beta2, w.eps, stream=stream)
         # at least three warm-up steps: the first selections run the dense passes, the threshold prediction
         # carries the rest
         for t in range(max(args.warmup, 3)):
-            opt.step(ring[t % 2], theta)
+            opt.step(feed(t), theta)
         opt.check_status()
         st0 = opt.buffer("status").cpu().tolist()
         opt.set_profiling(["topk_sweep"])
@@ -411,7 +449,7 @@ def main():
         start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         start.record(stream)
         for t in range(args.steps):
-            opt.step(ring[(args.warmup + t) % 2], theta)
+            opt.step(feed(args.warmup + t), theta)
         stop.record(stream)
         replicas.barrier(dist)
         clocks = sampler.stop()
@@ -442,7 +480,7 @@ def main():
         # ---- per-kernel breakdown of the step, from a few extra steps with an event pair around every launch
         opt.set_profiling(KERNELS["topk"])
         for t in range(3):
-            opt.step(ring[(args.warmup + args.steps + t) % 2], theta)  # the ring goes on in step
+            opt.step(feed(args.warmup + args.steps + t), theta)  # the gradients go on in step
         per_kernel = {}
         for k in KERNELS["topk"]:
             ms, cnt = opt.kernel_time(k)
@@ -455,14 +493,13 @@ def main():
             "ms_per_step": ms_per_step, "steps_per_s": 1e3 / ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(pt),
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "kernels": per_kernel,
+            "gradients": feed.kind,
             "status": {"word": st1[0], "dense": st1[1] - st0[1], "candidate": st1[2] - st0[2],
                        "gave_up": [st1[k] - st0[k] for k in (3, 4, 5, 6)]},
         }
 
         # ---- end to end through the C ABI with HOST buffers (copies inside the timed region)
         if not args.no_e2e:
-            del ring[1]
-            torch.cuda.empty_cache()
             hg = ht = None
             try:  # n d 4 bytes of pinned host memory per rank: every rank must get its own or all skip the leg
                 hg = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
@@ -471,7 +508,7 @@ def main():
             except RuntimeError:
                 ok = 0.0
             if -replicas.max_over_ranks(-ok, dist, device) > 0.5:
-                hg.copy_(ring[0])
+                hg.copy_(feed(0))
                 ht.copy_(theta)
                 opt.step_host(hg, ht)  # allocates the staging buffers outside the timed region
                 replicas.barrier(dist)
@@ -490,11 +527,11 @@ def main():
 
         # ---- the oracle on the host cores, rank 0 at N = 1 only
         if rank == 0 and world == 1 and not args.no_cpu_baseline:
-            v, cores, what, dt, _ = oracle_sample(pt, ring[0], budget_s=20.0)
+            v, cores, what, dt, _ = oracle_sample(pt, feed(0), budget_s=20.0)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "ms_per_step": dt * 1e3,
                                     "sample": what}
         opt.close()
-        del ring, theta
+        del feed, theta
         torch.cuda.empty_cache()
 
     # ---- every configuration, one compressor per number (rank 0 at N = 1 only)
@@ -507,8 +544,8 @@ def main():
                                       cache))
         cache.clear()
         line["configs"] = entries
-        line["configs_protocol"] = ("per entry: %d steps between two CUDA events after %d warm-up steps, ring of 2 gradient "
-                                    "batches; min_bytes = (12 n + 32) d with error feedback ((10 n + 32) d with bfloat16 "
+        line["configs_protocol"] = ("per entry: %d steps between two CUDA events after %d warm-up steps, a different "
+                                    "gradient batch every step (each entry's `gradients`); min_bytes = (12 n + 32) d with error feedback ((10 n + 32) d with bfloat16 "
                                     "gradients), (4 n + 32) d for k = d" % (args.config_steps, args.config_warmup))
     if rank == 0:
         print(json.dumps(line))

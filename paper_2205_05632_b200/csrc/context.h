@@ -52,6 +52,8 @@ struct SegState {
     uint32_t sel_ready;   // multi-CTA select: the threshold bin has been found, the emit kernel may run
     uint32_t boost;       // the candidate margin is doubled this many times (raised when a list came up short)
     uint32_t streak;      // selections decided inside the list since the margin last changed
+    uint32_t hold;        // a doubling is taken back after 32 << hold such selections in a row
+    uint32_t probing;     // 1: the margin was last changed by taking a doubling back
 };
 
 // Block / tile tables shared by the tiled kernels (device pointers).

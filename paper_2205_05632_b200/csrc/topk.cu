@@ -281,22 +281,35 @@ __device__ __forceinline__ void predict_next(SegState* st, uint32_t tau, uint32_
 // How many candidates the next step's predicted threshold should let through for a segment that keeps kb: the
 // count of keys above a fixed threshold moves by about sqrt(kb) from one step to the next (eight of those are
 // allowed for), plus a quarter of kb for drift of the gradient scale. A segment whose list came up short gets
-// its margin doubled (`boost` times, at most three); the doubling is taken back one step at a time after 32
-// selections in a row were decided inside the list. Long lists thus carry about 1.26 kb entries, short ones
+// its margin doubled (`boost` times, at most three); the doubling is taken back one step at a time after enough
+// selections in a row were decided inside the list (margin_held). Long lists thus carry about 1.26 kb entries, short ones
 // (kb = 50: 170) proportionally more.
 __device__ __forceinline__ uint32_t want_candidates(uint32_t kb, uint32_t boost) {
     const uint32_t margin = ((kb >> 2) + (uint32_t)(8.0f * sqrtf((float)kb)) + 32u) << (boost < 3u ? boost : 3u);
     const uint32_t most = 4u * kb + 512u;  // half the list's capacity
     return kb + (margin < most - kb ? margin : most - kb);
 }
+// Taking a doubling back is a probe: if the smaller margin comes up short (a dense-pass step, which costs several
+// ordinary steps), the margin was needed, and the next probe waits twice as long (32, 64, ... 32768 selections). A
+// probe that holds for a whole waiting time halves the wait again. Gradients that alternate between two levels
+// need the first doubling for good: with a fixed wait of 32 every 33rd step ran the dense passes (n = 32,
+// d = 2^27: 9.1 -> 9.6 ms per step on average).
+constexpr uint32_t kHoldMax = 10u;
 __device__ __forceinline__ void margin_came_up_short(SegState* st) {
     if (st->boost < 3u) ++st->boost;
+    if (st->probing && st->hold < kHoldMax) ++st->hold;
+    st->probing = 0u;
     st->streak = 0u;
 }
 __device__ __forceinline__ void margin_held(SegState* st) {
-    if (++st->streak >= 32u) {
+    if (++st->streak >= (32u << st->hold)) {
         st->streak = 0u;
-        if (st->boost) --st->boost;
+        if (st->probing && st->hold) --st->hold;
+        st->probing = 0u;
+        if (st->boost) {
+            --st->boost;
+            st->probing = 1u;
+        }
     }
 }
 
@@ -1012,6 +1025,28 @@ __device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b
                     st->edge = (uint32_t)(NBINS - 1 - ((int)threadIdx.x * PER + j)) << 20;
                 running += cnt[j];
             }
+        }
+    }
+    if (PASS == 2) {
+        // Pass 1 places that edge on a grid of an eighth of a binade. Under error feedback the magnitudes pile up
+        // just below the threshold (a coordinate grows until it is kept), so a bin edge a few per cent below the
+        // threshold can let through many times the wanted number, more than the list holds, and the segment came
+        // back to the dense passes step after step. When the wanted number is reached inside the threshold's own
+        // pass-1 bin, this pass places the edge 1024 times finer; when that bin and the bins above hold fewer than
+        // wanted but at least half the margin, the bin's lower edge is taken rather than one further down.
+        const uint32_t want = want_candidates(kb, st->boost);
+        const uint32_t above = kb - k_rem;     // keys in the pass-1 bins above the threshold's
+        const uint32_t want2 = want - above;   // want > kb > above
+        if (excl < want2 && want2 <= incl) {
+            uint32_t running = excl;
+#pragma unroll
+            for (int j = 0; j < PER; ++j) {
+                if (running < want2 && want2 <= running + cnt[j])
+                    st->edge = (prefix << 20) | ((uint32_t)(NBINS - 1 - ((int)threadIdx.x * PER + j)) << 10);
+                running += cnt[j];
+            }
+        } else if (threadIdx.x == 0 && total < want2 && above + total >= kb + ((want - kb) >> 1)) {
+            st->edge = prefix << 20;
         }
     }
     if (threadIdx.x == 0 && total < k_rem) atomicOr(b.status, 2u);

@@ -128,6 +128,23 @@ class Workload:
         return G
 
 
+def iid_normal(w: Workload) -> bool:
+    """True when every coordinate of every row is an independent N(0,1) draw (one block, no per-tensor scale)."""
+    return w._row is _row_normal and len(w.block_offsets) == 2
+
+
+def grads_with_tail(w: Workload, extra: int) -> torch.Tensor:
+    """For iid_normal workloads: one flat tensor of n*d + extra draws. Every window [o, o + n*d) of it, viewed as
+    [n, d], is a gradient batch of the workload's distribution, and windows at different offsets give a coordinate
+    independent values: a fresh batch per step out of one buffer."""
+    assert iid_normal(w) and w._gen is not None
+    flat = torch.empty(w.n * w.d + extra, device=w.device, dtype=torch.float32)
+    for i in range(w.n):
+        flat[i * w.d:(i + 1) * w.d] = _row_normal(w)
+    flat[w.n * w.d:] = torch.randn(extra, generator=w._gen, device=w.device, dtype=torch.float32)
+    return flat
+
+
 def _row_normal(w: Workload) -> torch.Tensor:
     return torch.randn(w.d, generator=w._gen, device=w.device, dtype=torch.float32)
 

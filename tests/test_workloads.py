@@ -46,3 +46,19 @@ def test_config3_has_exact_zeros():
     g = w.grads()
     frac = float((g == 0).float().mean())
     assert 0.045 < frac < 0.055
+
+
+def test_windows_over_one_buffer_are_fresh_batches():
+    """grads_with_tail: the head is the batch grads() would have drawn, every window is N(0,1) and two windows
+    give a coordinate unrelated values; workloads with per-tensor scales or several blocks are refused."""
+    a, b = W.config1(), W.config1()
+    a.start(), b.start()
+    assert W.iid_normal(a) and not W.iid_normal(W.config3(0.01)) and not W.iid_normal(W.config4(W.TOPK))
+    extra = 64 * 5
+    flat = W.grads_with_tail(a, extra)
+    assert flat.shape == (4 * 65536 + extra,)
+    assert torch.equal(flat[:4 * 65536].view(4, 65536), b.grads())
+    w0 = flat[0:4 * 65536].view(4, 65536)
+    w1 = flat[64:64 + 4 * 65536].view(4, 65536)
+    assert abs(float(w1.mean())) < 0.01 and abs(float(w1.std()) - 1.0) < 0.01
+    assert abs(float((w0 * w1).mean())) < 0.01  # no correlation between what a coordinate sees in two steps
