@@ -67,7 +67,7 @@ def measured_peak_gbs():
 # space aside) at the time of the capture: once the code changes the figure no longer describes the kernel and
 # None is reported.
 TRAFFIC_PER_ELEM = {
-    "topk_sweep": (1600309760 / 134217728, "topk.cu", "0732a97b1bd3ea21"),
+    "topk_sweep": (1599850752 / 134217728, "topk.cu", "f7c17c2f5421d19c"),
 }
 
 
@@ -231,11 +231,13 @@ class GradientFeed:
     draw each step, and the rows keep their alignment; otherwise (no such workload exists among the entries) a
     ring of as many batches as fit, at least two."""
 
+    batches = FEED_RING  # --feed-ring
+
     def __init__(self, w, bf16=False):
         per = w.n * w.d * 4
         self.n, self.d, self.flat, self.ring = w.n, w.d, None, None
-        if FEED_RING * per <= FEED_RING_BYTES or not W.iid_normal(w):
-            count = max(2, min(FEED_RING, FEED_RING_BYTES // per))
+        if GradientFeed.batches * per <= FEED_RING_BYTES or not W.iid_normal(w):
+            count = max(2, min(GradientFeed.batches, FEED_RING_BYTES // per))
             self.ring = [w.grads() for _ in range(count)]
             if bf16:
                 self.ring = [g.bfloat16() for g in self.ring]
@@ -409,7 +411,10 @@ def main():
     ap.add_argument("--config-steps", type=int, default=20)
     ap.add_argument("--config-warmup", type=int, default=40)
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--feed-ring", type=int, default=FEED_RING,
+                    help="gradient batches prepared per entry (profiler captures of small cases use 2 to hold less memory)")
     args = ap.parse_args()
+    GradientFeed.batches = max(2, args.feed_ring)
 
     if args.impl == "reference":
         run_reference(args)
