@@ -352,6 +352,59 @@ def test_topk_candidate_path_survives_gradients_that_alternate_between_two_batch
         p.close()
 
 
+@pytest.mark.parametrize("blocks", [1, 24])
+def test_topk_dense_passes_stay_rare_over_hundreds_of_alternating_steps(blocks):
+    # Two alternating batches over 400 steps: under error feedback the threshold then swings between two levels
+    # and the magnitudes pile up just below it. A smaller candidate margin is probed again and again; a probe that
+    # fails costs a dense-pass step, so failed probes must back off, and a segment sent to the dense passes must
+    # come back with a threshold fine enough not to return there on the next step.
+    n, d = 4, 48 * 8192
+    offs = [d // blocks * b for b in range(blocks)] + [d]
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    ring = [torch.randn(n, d, generator=gen, device="cuda") for _ in range(2)]
+    theta = torch.zeros(d, device="cuda")
+    opt = CompAMS(n, d, offs, TOPK, 0.01)
+    try:
+        steps, after = 400, 8
+        for t in range(steps):
+            if t == after:
+                st0 = _status(opt)
+            opt.step(ring[t % 2], theta)
+        st = _status(opt)
+        opt.check_status()
+        selections = (steps - after) * n * blocks
+        assert (st[1] - st0[1]) + (st[2] - st0[2]) == selections
+        dense = st[1] - st0[1]
+        # a fixed wait of 32 selections between probes gives one dense-pass selection in 33: 3 %
+        assert dense <= 0.015 * selections, "dense passes decided %d of %d selections: %r" % (dense, selections, st)
+    finally:
+        opt.close()
+
+
+def test_topk_no_dense_pass_after_the_first_steps_with_a_new_batch_every_step():
+    # independent gradients every step, 300 steps, a long list (slices) and short ones (one CTA each): once the
+    # error accumulators have filled, every selection is decided inside its candidate list, through every change
+    # of the candidate margin
+    n, d = 4, 1 << 22
+    offs = [0, 1 << 21, (1 << 21) + 300000, d]
+    gen = torch.Generator(device="cuda").manual_seed(12)
+    theta = torch.zeros(d, device="cuda")
+    G = torch.empty(n, d, device="cuda")
+    opt = CompAMS(n, d, offs, TOPK, 0.01)
+    try:
+        steps, after = 300, 40
+        for t in range(steps):
+            if t == after:
+                st0 = _status(opt)
+            G.normal_(generator=gen)
+            opt.step(G, theta)
+        st = _status(opt)
+        opt.check_status()
+        assert st[2] - st0[2] == (steps - after) * n * 3 and st[1] == st0[1], "dense passes after step %d: %r -> %r" % (after, st0, st)
+    finally:
+        opt.close()
+
+
 def test_topk_prediction_failures_fall_back_exactly():
     # the gradient scale jumps by orders of magnitude between steps: too few candidates, too many,
     # thresholds far above the predicted range - every case must still give the exact Top-k
