@@ -961,6 +961,8 @@ __device__ __forceinline__ void dense_hist(const Tables& t, const TopkBuffers& b
     }
 }
 
+constexpr int kLowBins = 64;  // fine bins at the bottom of the threshold's pass-1 bin that give the density there
+
 template <int NBINS, int BITS, int PASS>
 __device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b, size_t sg, uint32_t* scratch) {
     constexpr int PER = NBINS / kThreads;
@@ -1027,13 +1029,13 @@ __device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b
             }
         }
     }
-    if (PASS == 2) {
+    if constexpr (PASS == 2) {
         // Pass 1 places that edge on a grid of an eighth of a binade. Under error feedback the magnitudes pile up
         // just below the threshold (a coordinate grows until it is kept), so a bin edge a few per cent below the
         // threshold can let through many times the wanted number, more than the list holds, and the segment came
         // back to the dense passes step after step. When the wanted number is reached inside the threshold's own
         // pass-1 bin, this pass places the edge 1024 times finer; when that bin and the bins above hold fewer than
-        // wanted but at least half the margin, the bin's lower edge is taken rather than one further down.
+        // wanted, the edge is extrapolated below the bin's lower edge (see there).
         const uint32_t want = want_candidates(kb, st->boost);
         const uint32_t above = kb - k_rem;     // keys in the pass-1 bins above the threshold's
         const uint32_t want2 = want - above;   // want > kb > above
@@ -1045,8 +1047,19 @@ __device__ __forceinline__ void dense_find(const Tables& t, const TopkBuffers& b
                     st->edge = (prefix << 20) | ((uint32_t)(NBINS - 1 - ((int)threadIdx.x * PER + j)) << 10);
                 running += cnt[j];
             }
-        } else if (threadIdx.x == 0 && total < want2 && above + total >= kb + ((want - kb) >> 1)) {
-            st->edge = prefix << 20;
+        } else if (total < want2 && threadIdx.x == kThreads - 1 - kLowBins / PER) {
+            // The wanted count is reached below the threshold's pass-1 bin (the threshold sits just above a bin
+            // boundary): the edge goes below the boundary by as far as the missing candidates need at the density
+            // of the bin's lowest kLowBins fine bins. Further down the density only grows, so at least the wanted
+            // number comes through, and far fewer than down to the next boundary. This thread's bins end where
+            // those fine bins begin: `incl` counts everything above them.
+            const uint32_t low = total - incl;
+            if (low) {
+                const unsigned long long ext = (unsigned long long)(want2 - total) * ((unsigned long long)kLowBins << 10) / low;
+                const uint32_t top = prefix << 20;
+                const uint32_t fine = ext < (unsigned long long)top ? top - (uint32_t)ext : 0u;
+                if (fine > st->edge) st->edge = fine;  // never below the pass-1 edge, which is known to suffice
+            }
         }
     }
     if (threadIdx.x == 0 && total < k_rem) atomicOr(b.status, 2u);
