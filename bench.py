@@ -65,20 +65,27 @@ def measured_peak_gbs():
 # kernel, from an ncu capture of a smaller case of the same kernel (d = 2^24, n = 8; the traffic of these
 # streaming kernels grows in proportion to n d), with a hash of the kernel's source code (comments and white
 # space aside) at the time of the capture: once the code changes the figure no longer describes the kernel and
-# None is reported.
+# None is reported. The kernel's code is the stretch of its file between the two markers (the kernel with the
+# device functions it alone uses) plus the shared helper header.
 TRAFFIC_PER_ELEM = {
-    "topk_sweep": (1599850752 / 134217728, "topk.cu", "f7c17c2f5421d19c"),
+    "topk_sweep": (1599850752 / 134217728, "topk.cu", ("constexpr uint32_t kNothingKept", "void predict_next("),
+                   "b1b2c4af58fd5755"),
 }
 
 
-def code_hash(paths):
-    """Hash of the concatenated sources with comments removed and white space collapsed."""
+def code_hash(paths, between=None):
+    """Hash of the concatenated sources with comments removed and white space collapsed; of the first file only
+    the stretch from the first marker of `between` up to the second."""
     import hashlib
     import re
     text = ""
-    for p in paths:
+    for k, p in enumerate(paths):
         with open(p) as f:
-            text += f.read()
+            part = f.read()
+        if k == 0 and between is not None:
+            a = part.index(between[0])
+            part = part[a:part.index(between[1], a)]
+        text += part
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     text = re.sub(r"//[^\n]*", "", text)
     text = re.sub(r"\s+", " ", text)
@@ -88,11 +95,11 @@ def code_hash(paths):
 def captured_traffic(kernel: str, elems: int):
     if kernel not in TRAFFIC_PER_ELEM:
         return None
-    per_elem, src, want = TRAFFIC_PER_ELEM[kernel]
+    per_elem, src, between, want = TRAFFIC_PER_ELEM[kernel]
     base = os.path.join(ROOT, "paper_2205_05632_b200", "csrc")
     try:
-        have = code_hash([os.path.join(base, src), os.path.join(base, "common.cuh")])
-    except OSError:
+        have = code_hash([os.path.join(base, src), os.path.join(base, "common.cuh")], between)
+    except (OSError, ValueError):
         return None
     return int(per_elem * elems) if have == want else None
 
