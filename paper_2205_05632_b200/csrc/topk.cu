@@ -313,6 +313,15 @@ __device__ __forceinline__ void margin_held(SegState* st) {
     }
 }
 
+// After a selection decided inside its list of c candidates: a list that held by less than a quarter of its margin
+// was a near miss and is treated like a list that came up short, only without the dense passes (thresholds that
+// swing from step to step announce themselves this way: d = 2^24, n = 8, two alternating batches: 1.01 k_b
+// candidates a dozen steps before 0.94 k_b).
+__device__ __forceinline__ void margin_after_selection(SegState* st, uint32_t kb, uint32_t c) {
+    if (c - kb < (want_candidates(kb, st->boost) - kb) >> 2) margin_came_up_short(st);
+    else margin_held(st);
+}
+
 constexpr int kSelUnroll = 4;   // candidate loads in flight per thread while scanning a list
 // One CTA per short list, 2048 threads to the SM at 32 registers. 1024 threads per list keep enough loads in flight
 // to finish one list soonest (few lists: d = 2^20, n = 8: step 0.051 ms against 0.058 with 512); with more lists
@@ -573,7 +582,7 @@ __global__ void __launch_bounds__(NT, 2048 / NT) topk_select_kernel(Tables t, To
             edge = tau_hat > gap ? tau_hat - gap : 0u;
         }
         predict_next(st, tau, edge, true);
-        margin_held(st);
+        margin_after_selection(st, kb, c);
         st->fallback = 0u;
         atomicAdd(b.status + 2, 1u);  // selections decided inside their candidate list
     }
@@ -911,7 +920,7 @@ __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBu
             edge = tau_hat > gap ? tau_hat - gap : 0u;
         }
         predict_next(st, tau, edge, true);
-        margin_held(st);
+        margin_after_selection(st, kb, c);
         st->fallback = 0u;
         atomicAdd(b.status + 2, 1u);  // selections decided inside their candidate list
     }
