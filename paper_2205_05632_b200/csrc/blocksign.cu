@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(kThreads, sizeof(GT) == 2 ? COMPAMS_BF16_SWEEP
                                                                int deferred, const __grid_constant__ SegParams sp_) {
     __shared__ double red[kWarps];
     __shared__ uint32_t sh_first[kWarps];
-    dependency_wait();  // on small problems launched as a programmatic dependent of the step before (whose server
+    dependency_wait();  // while n d <= kChainMaxElems launched as a programmatic dependent of the step before (whose server
                         // kernel still reads the sign words this kernel is about to overwrite)
     allow_dependents();
     const int tile = blockIdx.x;
@@ -447,7 +447,7 @@ static BsBuffers own_rows(const compams_context* c) {
 
 cudaError_t launch_bs_sweep(compams_context* c, const void* grads) {
     dim3 grid((unsigned)c->tab.ntiles, (unsigned)c->n);
-    if (c->chain) {  // small problem: the launch overlaps the tail of whatever kernel precedes it on the stream
+    if (c->chain) {  // n d <= kChainMaxElems: the launch overlaps the tail of whatever kernel precedes it on the stream
         if (c->grad_bf16)
             return counted(c, launch_after(bs_sweep_kernel<bf16_bits>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c),
                                 (const bf16_bits*)grads, c->e_is_x ? 1 : 0, c->segp));

@@ -10,7 +10,7 @@
 #include "common.cuh"
 
 #ifndef COMPAMS_CHAIN_MAX
-#define COMPAMS_CHAIN_MAX ((int64_t)1 << 25)
+#define COMPAMS_CHAIN_MAX ((int64_t)1 << 28)
 #endif
 
 namespace compams {
@@ -118,7 +118,7 @@ struct compams_context {
     int32_t n_total = 0;  // workers the server averages over (> n when the workers are sharded over several handles)
     int32_t row0 = 0;     // index of this handle's first worker among the n_total
     int64_t d = 0;
-    bool chain = false;      // small problem: the Top-k kernels of a step are launched as programmatic dependents
+    bool chain = false;      // n d <= kChainMaxElems: the kernels of a step are launched as programmatic dependents
     bool grad_bf16 = false;  // the gradients of the call being enqueued are bfloat16 (16-bit patterns), not fp32
     int32_t M = 0;
     int32_t compressor = 0;

@@ -208,7 +208,7 @@ __device__ __forceinline__ void topk_sweep_tile_bf16x8(const bf16_bits* __restri
 template <typename GT>
 __global__ void __launch_bounds__(kThreads, sizeof(GT) == 2 ? COMPAMS_BF16_TOPK_SWEEP_CTAS : 6) topk_sweep_kernel(Tables t, TopkBuffers b, const GT* __restrict__ G,
                                                                  const __grid_constant__ SegParams sp_) {
-    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    dependency_wait();   // launched as a programmatic dependent while n d <= kChainMaxElems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint2 sh_cand[kTileCand];
     __shared__ uint32_t sh_cnt, sh_base;
@@ -388,7 +388,7 @@ __device__ __forceinline__ uint32_t offset_digit(uint32_t xbits, uint32_t tau_ha
 template <int NT>
 __global__ void __launch_bounds__(NT, 2048 / NT) topk_select_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                int nlist) {
-    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    dependency_wait();   // launched as a programmatic dependent while n d <= kChainMaxElems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint32_t local[kSelBins];  // histogram of the list
     __shared__ uint2 surv[kSurvCap];
@@ -600,7 +600,7 @@ __global__ void __launch_bounds__(NT, 2048 / NT) topk_select_kernel(Tables t, To
 
 __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                 int nlist, int parts) {
-    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    dependency_wait();   // launched as a programmatic dependent while n d <= kChainMaxElems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint32_t local[kSelBins];
     __shared__ uint32_t scratch[kWarps];
@@ -699,7 +699,7 @@ __global__ void __launch_bounds__(kThreads) topk_selhist_kernel(Tables t, TopkBu
 
 __global__ void __launch_bounds__(kThreads) topk_selemit_kernel(Tables t, TopkBuffers b, const int32_t* __restrict__ seg_list,
                                                                 int nlist, int parts) {
-    dependency_wait();   // launched as a programmatic dependent on small problems: the kernel before must be done
+    dependency_wait();   // launched as a programmatic dependent while n d <= kChainMaxElems: the kernel before must be done
     allow_dependents();  // ... and the next one may move in behind this one's last wave
     __shared__ uint2 surv[kSurvSmem];
     __shared__ uint32_t sh_hist[kThreads];
@@ -1421,7 +1421,7 @@ cudaError_t launch_topk_sweep(compams_context* c, const void* grads) {
     return counted(c, cudaGetLastError());
 }
 
-// On small problems the kernels of a step are launched as programmatic dependents of one another (each
+// While n d <= kChainMaxElems the kernels of a step are launched as programmatic dependents of one another (each
 // waits for its predecessor before its first global access): the launch latency and the prologue of a
 // kernel then overlap the tail of the one before, which is most of what such a step costs.
 template <typename... KArgs, typename... Args>
