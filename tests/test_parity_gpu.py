@@ -405,6 +405,25 @@ def test_topk_no_dense_pass_after_the_first_steps_with_a_new_batch_every_step():
         opt.close()
 
 
+@pytest.mark.parametrize("name,n,blocks,block_len,ring,steps", [
+    ("one block, two alternating batches", 4, 1, 48 * 8192 + 77, 2, 100),
+    ("24 blocks, two alternating batches", 3, 24, 20000, 2, 100),
+    ("one block, a new batch every step", 4, 1, 40 * 8192 + 5, 0, 80),
+    ("720 lists layer-wise", 8, 90, 9000, 2, 40)])
+def test_topk_long_chained_runs_against_the_oracle(name, n, blocks, block_len, ring, steps):
+    # long enough for the candidate margin to be raised, probed and taken back several times (alternating batches
+    # make lists come up short and nearly short), and with enough lists for the narrower select CTAs: every step
+    # against the oracle, E on every seventh
+    d = blocks * block_len
+    offs = [block_len * b for b in range(blocks + 1)]
+    gen0 = torch.Generator(device="cuda").manual_seed(77)
+    batches = [torch.randn(n, d, generator=gen0, device="cuda") for _ in range(ring)]
+
+    def make(gen, t):
+        return batches[t % ring] if ring else torch.randn(n, d, generator=gen, device="cuda")
+    _pair_run(n, d, offs, TOPK, 0.01, make, steps=steps, check_e_every=7)
+
+
 def test_topk_prediction_failures_fall_back_exactly():
     # the gradient scale jumps by orders of magnitude between steps: too few candidates, too many,
     # thresholds far above the predicted range - every case must still give the exact Top-k
