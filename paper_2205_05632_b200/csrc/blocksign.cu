@@ -221,27 +221,42 @@ __global__ void __launch_bounds__(kThreads, sizeof(GT) == 2 ? COMPAMS_BF16_SWEEP
     }
 }
 
-// One CTA per (worker, block): scale = ||x_B||_1 / d_B from the tile sums (Definition 2).
-__global__ void __launch_bounds__(kThreads) bs_scales_kernel(Tables t, BsBuffers b) {
-    __shared__ double red[kWarps];
+// One CTA per (worker, block): scale = ||x_B||_1 / d_B from the tile sums (Definition 2). Built for 256 threads
+// (many blocks of a few tiles) and for 1024 with four tile sums requested at a time (a whole-vector block has
+// thousands of tiles and only n CTAs to add them: 256 threads took 33 us at d = 2^26, n = 8, most of it waiting
+// for one load after the other). The order of the additions is fixed by the tile count and the thread count,
+// and every handle of a sharded run makes the same choice, so equal inputs give equal bits.
+template <int NT>
+__global__ void __launch_bounds__(NT) bs_scales_kernel(Tables t, BsBuffers b) {
+    __shared__ double red[NT / 32];
     allow_dependents();
     dependency_wait();  // the sweep's tile sums and word shares
     const int blk = blockIdx.x, i = blockIdx.y;
     const SegInfo* si = t.segs + blk;
     const double* ts = b.tile_sum + (size_t)i * t.ntiles + si->tile0;
+    const int nt = si->ntile_b;
     double part = 0.0;
-    for (int k = threadIdx.x; k < si->ntile_b; k += kThreads) part += ts[k];
+    int k = threadIdx.x;
+    for (; k + 3 * NT < nt; k += 4 * NT) {
+        const double s0 = ts[k], s1 = ts[k + NT], s2 = ts[k + 2 * NT], s3 = ts[k + 3 * NT];
+        part += s0;
+        part += s1;
+        part += s2;
+        part += s3;
+    }
+    for (; k < nt; k += NT) part += ts[k];
     // the sign word two neighbouring tiles have in common: one share from each
     {
         const uint2* ed = b.edge + (size_t)i * t.ntiles + si->tile0;
         const int wb = (si->len + 31) >> 5;
         uint32_t* words = b.bits + (size_t)i * (size_t)b.W + (size_t)b.word_off[blk];
-        for (int k = threadIdx.x; k < si->ntile_b; k += kThreads) {
-            const int q = (k + 1) * (kTile / 32) - 1;
-            if (q < wb) words[q] = ed[k].y | (k + 1 < si->ntile_b ? ed[k + 1].x : 0u);
+#pragma unroll 4
+        for (int j = threadIdx.x; j < nt; j += NT) {
+            const int q = (j + 1) * (kTile / 32) - 1;
+            if (q < wb) words[q] = ed[j].y | (j + 1 < nt ? ed[j + 1].x : 0u);
         }
     }
-    const double S = block_sum_double(part, red);
+    const double S = block_sum_double<NT / 32>(part, red);
     // one division in binary64, one rounding to fp32
     if (threadIdx.x == 0) b.scales_cur[(size_t)i * t.M + blk] = __double2float_rn(S / (double)si->len);
 }
@@ -465,7 +480,9 @@ cudaError_t launch_bs_sweep(compams_context* c, const void* grads) {
 
 cudaError_t launch_bs_scales(compams_context* c) {
     dim3 grid((unsigned)c->M, (unsigned)c->n);
-    return counted(c, launch_after(bs_scales_kernel, grid, dim3(kThreads), c->stream, c->tab, own_rows(c)));
+    if (c->tab.ntiles > 256 * (int64_t)c->M)  // on average more than 256 tiles to a block
+        return counted(c, launch_after(bs_scales_kernel<1024>, grid, dim3(1024), c->stream, c->tab, own_rows(c)));
+    return counted(c, launch_after(bs_scales_kernel<kThreads>, grid, dim3(kThreads), c->stream, c->tab, own_rows(c)));
 }
 
 cudaError_t launch_bs_apply(compams_context* c, float* theta) {

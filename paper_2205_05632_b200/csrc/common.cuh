@@ -239,7 +239,8 @@ __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t x, uint32_t* s
 }
 
 // Deterministic CTA sum of one double per thread (fixed shuffle tree, then warps in order).
-// Result valid in thread 0. `scratch` holds kWarps doubles.
+// Result valid in thread 0. `scratch` holds one double per warp of the CTA (WARPS of them).
+template <int WARPS = kWarps>
 __device__ __forceinline__ double block_sum_double(double x, double* scratch) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -250,7 +251,7 @@ __device__ __forceinline__ double block_sum_double(double x, double* scratch) {
     double s = 0.0;
     if (threadIdx.x == 0) {
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) s += scratch[w];
+        for (int w = 0; w < WARPS; ++w) s += scratch[w];
     }
     return s;
 }
